@@ -1,0 +1,190 @@
+/*
+ * mqa_decode.h - C ABI of the B200 (sm_100a) multiquery decode-attention library.
+ *
+ * Operation ("Efficiently Scaling Transformer Inference", Section 3.3): in
+ * multiquery attention every sequence has n_heads query heads but a single key
+ * head and a single value head that all query heads share.  In the generate
+ * phase there is one query token per sequence, attending to that sequence's
+ * whole KV cache; the step's cost is reading the cache from HBM once
+ * (Section 2, "Memory costs"; Section 2.1).  For every sequence b and head h:
+ *
+ *     out[b,h,:] = sum_{l < lengths[b]} softmax_l( scale * q[b,h,:].k[b,l,:] ) * v[b,l,:]
+ *
+ * The kernels read each K/V tile once and use it for all H heads, evaluate the
+ * softmax in base 2 (Section 3.5 names base-2 softmax as an implementation
+ * choice; the function is the same), split the sequence axis across thread
+ * blocks with running-max partial results, and merge the partials with a
+ * log-sum-exp combine.
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer unless the parameter name ends in _host.
+ *   - Layouts are row-major and dense: q [B,H,D], k_cache/v_cache [B,Lmax,D],
+ *     out [B,H,D], lengths [B].  q/k/v are bf16, out is fp32, lengths int32.
+ *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - Calls enqueue work on `stream` and return without synchronising, except
+ *     mqa_check_status and mqa_decode_host, which synchronise the stream.
+ *   - Inputs are read-only.  out is fully overwritten for every (b,h).
+ *   - lengths[b] counts the valid cache rows of sequence b (the current token's
+ *     K/V row already appended) and is clamped into [0, Lmax] on the device.
+ *     lengths[b] == 0 gives an all-zero output row.  Cache rows at or beyond
+ *     lengths[b] may hold any bits (NaN included); they never affect out.
+ *   - Every function that returns int returns an mqa_status_t.  On any error
+ *     nothing is launched.
+ *   - Same inputs and same plan give bit-identical output.
+ *   - Thread safety: concurrent calls are safe when they use different
+ *     workspaces.  Two calls sharing a workspace must be stream-ordered.
+ */
+#ifndef MQA_DECODE_H_
+#define MQA_DECODE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MQA_OK = 0,
+    MQA_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, bad plan field   */
+    MQA_ERR_UNSUPPORTED_SHAPE = 2,   /* D not in {64,128,256}, H > 64, tile count overflow */
+    MQA_ERR_MISALIGNED = 3,          /* q/k/v/out/workspace not 16-byte aligned            */
+    MQA_ERR_WORKSPACE_TOO_SMALL = 4,
+    MQA_ERR_ARCH = 5,                /* current device is not compute capability 10.x      */
+    MQA_ERR_CUDA = 6,                /* a CUDA runtime/driver call failed                  */
+    MQA_ERR_TIMEOUT = 7              /* a bounded device-side wait ran out (see check_status) */
+} mqa_status_t;
+
+/* Kernel families (mqa_plan_t.path). */
+enum {
+    MQA_PATH_AUTO = 0,
+    MQA_PATH_FMA = 1,   /* fp32 FMA kernel, any supported shape                      */
+    MQA_PATH_TC = 2     /* tcgen05 tensor-core kernel with TMA staging: D in {128,256}, H >= 8 */
+};
+
+/*
+ * Execution plan: which kernel family, how many persistent thread blocks share
+ * the flattened list of K/V tiles, and the tile height in cache rows.  The
+ * sequence axis is split wherever a block's share of tiles ends, so the split
+ * count per sequence follows from (B, lengths, num_ctas).
+ */
+typedef struct {
+    int path;        /* MQA_PATH_FMA or MQA_PATH_TC (AUTO only as a request)  */
+    int num_ctas;    /* 1 .. MQA_MAX_CTAS                                      */
+    int tile_rows;   /* cache rows per tile: 64 (FMA) or 128 (TC)              */
+} mqa_plan_t;
+
+#define MQA_MAX_CTAS 592          /* upper bound on mqa_plan_t.num_ctas (4 per SM on 148 SMs) */
+#define MQA_MAX_HEADS 64
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* mqa_status_string(int status);
+
+/*
+ * Bytes of device workspace mqa_decode needs for this shape under ANY plan the
+ * library may choose: a 256-byte header (device status word, tile total), one
+ * 8-byte record per sequence, and two partial-result slots per thread block
+ * (per slot: running max and running sum per head, and the unnormalised fp32
+ * accumulator [H,D]).  Returns 0 for an unsupported shape.  Host-only; no
+ * device is touched.
+ */
+size_t mqa_decode_workspace_bytes(int B, int H, int D, int Lmax);
+
+/*
+ * Zero the workspace header (the device status word).  Call once after
+ * allocating the workspace, before the first mqa_decode that uses it.
+ */
+int mqa_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The heuristic's plan for a shape on the current device (reads the SM count;
+ * falls back to 148 if no device is present).  Host-only otherwise.
+ * `requested_path` is MQA_PATH_AUTO, MQA_PATH_FMA or MQA_PATH_TC; a path the
+ * shape does not support gives MQA_ERR_UNSUPPORTED_SHAPE.
+ */
+int mqa_decode_plan(int B, int H, int D, int Lmax, int requested_path, mqa_plan_t* plan);
+
+/*
+ * One decode-attention step (Section 3.3; formula at the top of this file).
+ *   q          device bf16  [B,H,D]      16-byte aligned
+ *   k_cache    device bf16  [B,Lmax,D]   16-byte aligned
+ *   v_cache    device bf16  [B,Lmax,D]   16-byte aligned
+ *   lengths    device int32 [B]          read on the device only
+ *   out        device fp32  [B,H,D]      16-byte aligned, overwritten
+ *   scale      multiplies the fp32 logit (not folded into q)
+ *   workspace  device, 256-byte aligned, >= mqa_decode_workspace_bytes(...)
+ *   stream     cudaStream_t (NULL = legacy default stream)
+ * Supported: D in {64,128,256}; 1 <= H <= 64; B, Lmax >= 1 with
+ * B*ceil(Lmax/64) < 2^31.
+ */
+int mqa_decode(const void* q, const void* k_cache, const void* v_cache,
+               const int32_t* lengths, float* out,
+               int B, int H, int D, int Lmax, float scale,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same, with an explicit plan (tests and tuning). */
+int mqa_decode_with_plan(const void* q, const void* k_cache, const void* v_cache,
+                         const int32_t* lengths, float* out,
+                         int B, int H, int D, int Lmax, float scale,
+                         const mqa_plan_t* plan,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Same as mqa_decode_with_plan (plan == NULL selects the heuristic's plan), and
+ * additionally records `event_after_split` (a cudaEvent_t; may be NULL) on the
+ * stream between the split kernel and the combine kernel, so a benchmark can
+ * time the bandwidth-bound kernel on its own.
+ */
+int mqa_decode_profiled(const void* q, const void* k_cache, const void* v_cache,
+                        const int32_t* lengths, float* out,
+                        int B, int H, int D, int Lmax, float scale,
+                        const mqa_plan_t* plan,
+                        void* workspace, size_t workspace_bytes, void* stream,
+                        void* event_after_split);
+
+/*
+ * Synchronise `stream`, read the device status word from the workspace header,
+ * reset it to zero and return it (MQA_OK, or MQA_ERR_TIMEOUT if a bounded wait
+ * inside a kernel gave up; the output of that call is then undefined).
+ */
+int mqa_check_status(void* workspace, void* stream);
+
+/*
+ * Device scratch needed by mqa_decode_host: room for q, both caches, lengths,
+ * out (each rounded up to 256 bytes) plus mqa_decode_workspace_bytes.
+ */
+size_t mqa_decode_host_scratch_bytes(int B, int H, int D, int Lmax);
+
+/*
+ * End-to-end convenience call for HOST buffers (pinned memory recommended):
+ * copies q/k/v/lengths into `scratch` (device memory supplied by the caller),
+ * runs mqa_decode, copies out back to out_host and synchronises `stream`.
+ * The scratch header is initialised by this call.
+ */
+int mqa_decode_host(const void* q_host, const void* k_cache_host, const void* v_cache_host,
+                    const int32_t* lengths_host, float* out_host,
+                    int B, int H, int D, int Lmax, float scale,
+                    void* scratch, size_t scratch_bytes, void* stream);
+
+/* Number of kernels the last successful mqa_decode* call on this host thread
+ * launched (for launch accounting in benchmarks). */
+int mqa_last_launch_count(void);
+
+/*
+ * Host replay of the device tile schedule, for tests and tooling (no device is
+ * touched).  The K/V tiles of all sequences are numbered sequence-major and
+ * block `cta` of `num_ctas` takes a contiguous run of them; each piece of a
+ * sequence inside one run is a segment.  Writes up to max_segments records of
+ * 7 int32 each: {sequence, first tile, end tile (exclusive, both within the
+ * sequence), whole-sequence flag, partial slot (-1 if whole), owns-first-tile
+ * flag, block that owns the sequence's last tile}.  lengths_host is a HOST
+ * array.  Returns the number of segments of that block, or a negated
+ * mqa_status_t.
+ */
+int mqa_debug_schedule(const int32_t* lengths_host, int B, int Lmax, int tile_rows, int num_ctas, int cta,
+                       int32_t* records, int max_segments);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MQA_DECODE_H_ */

@@ -1,1 +1,5 @@
-"""B200-native multiquery decode attention over a KV cache (sm_100a)."""
+"""B200-native (sm_100a) multiquery decode attention over a KV cache.
+
+``binding`` wraps the C ABI of ``include/mqa_decode.h``; ``build`` compiles the
+CUDA sources in-tree; ``roofline`` holds the byte/flop accounting.
+"""

@@ -1,0 +1,183 @@
+// Shared device/host declarations of the multiquery decode-attention kernels:
+// workspace layout, the flattened tile schedule, and small helpers.
+//
+// Schedule.  Sequence b owns nt_b = ceil(len_b / tile_rows) tiles of its K/V
+// cache; the tiles of all sequences are numbered consecutively (sequence-major)
+// from 0 to T-1.  Persistent thread block i of G takes the contiguous run
+// [floor(i*T/G), floor((i+1)*T/G)).  A run crosses sequence boundaries; the
+// piece of a sequence inside one run is a "segment".  A segment that covers its
+// whole sequence writes the normalised output directly; any other segment
+// writes a partial result (running max m, running sum l, unnormalised
+// accumulator) into one of the block's two slots, and the combine kernel merges
+// the partial results of each cut sequence.  Each block recomputes the prefix
+// sums of the tile counts itself, so the host never reads `lengths`.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mqa {
+
+constexpr int kHeaderBytes = 256;
+constexpr int kMaxCtas = 592;
+constexpr int kMaxHeads = 64;
+
+// Workspace header words (int32).
+enum { kHdrStatus = 0, kHdrTotalTiles = 2, kHdrNumCtas = 3 };
+
+// Per-sequence record written by the block that owns the sequence's first tile.
+struct SeqInfo {
+    int first_slot;   // -1: the output was written directly; else slot index of the first partial
+    int last_cta;     // block that owns the sequence's last tile
+};
+
+__host__ __device__ inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// A partial-result slot: m[Hp4], l[Hp4], acc[H*D] (fp32), Hp4 = H rounded up to 4.
+__host__ __device__ inline size_t slot_floats(int H, int D) {
+    return (size_t)2 * round_up(H, 4) + (size_t)H * D;
+}
+__host__ __device__ inline size_t seqinfo_offset() { return kHeaderBytes; }
+__host__ __device__ inline size_t slots_offset(int B) {
+    return kHeaderBytes + ((size_t)B * sizeof(SeqInfo) + 255) / 256 * 256;
+}
+__host__ __device__ inline size_t workspace_bytes(int B, int H, int D) {
+    return slots_offset(B) + (size_t)2 * kMaxCtas * slot_floats(H, D) * sizeof(float);
+}
+
+struct Params {
+    const uint16_t* q;        // bf16 bits [B,H,D]
+    const uint16_t* k;        // [B,Lmax,D]
+    const uint16_t* v;        // [B,Lmax,D]
+    const int32_t* lengths;   // [B]
+    float* out;               // [B,H,D]
+    int B, H, D, Lmax;
+    float scale_log2;         // scale * log2(e): logits are kept in the base-2 domain
+    int tile_shift;           // log2(tile_rows)
+    int num_ctas;             // G
+    unsigned char* workspace;
+};
+
+__host__ __device__ __forceinline__ int clamp_len(int len, int Lmax) { return len < 0 ? 0 : (len > Lmax ? Lmax : len); }
+
+__device__ __forceinline__ int* ws_header(unsigned char* ws) { return reinterpret_cast<int*>(ws); }
+__device__ __forceinline__ SeqInfo* ws_seqinfo(unsigned char* ws) {
+    return reinterpret_cast<SeqInfo*>(ws + seqinfo_offset());
+}
+__device__ __forceinline__ float* ws_slot(unsigned char* ws, int B, int H, int D, int slot) {
+    return reinterpret_cast<float*>(ws + slots_offset(B)) + (size_t)slot * slot_floats(H, D);
+}
+
+// First tile of block i's run.
+__host__ __device__ inline long long span_begin(int i, int T, int G) { return (long long)i * T / G; }
+// The block whose run contains tile g (0 <= g < T).
+__host__ __device__ inline int cta_of_tile(long long g, int T, int G) {
+    return (int)(((g + 1) * G + T - 1) / T) - 1;
+}
+
+struct SchedShared {
+    int warp_sums[32];
+    int total;
+    int b0;         // sequence that contains the first tile of this block's run
+    int p0;         // global index of that sequence's first tile
+};
+
+// Block-wide: total tile count T, and (b0, p0) for the tile `g0 = span_begin(cta)`.
+// Every thread returns T; sh.b0/sh.p0 are valid after the call when the run is non-empty.
+template <int NTHREADS>
+__device__ inline int schedule_prologue(const int32_t* __restrict__ lengths, int B, int Lmax,
+                                        int tile_shift, int G, int cta, SchedShared& sh)
+{
+    const int tid = threadIdx.x;
+    const int tile_rows = 1 << tile_shift;
+    const int per = (B + NTHREADS - 1) / NTHREADS;
+    const int b_lo = min(B, tid * per), b_hi = min(B, b_lo + per);
+    int local = 0;
+    for (int b = b_lo; b < b_hi; ++b)
+        local += (clamp_len(lengths[b], Lmax) + tile_rows - 1) >> tile_shift;
+    // inclusive scan within the warp
+    int incl = local;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) sh.warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < NTHREADS / 32) ? sh.warp_sums[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        if (lane < NTHREADS / 32) sh.warp_sums[lane] = wi - w;   // exclusive warp offsets
+        if (lane == NTHREADS / 32 - 1) sh.total = wi;
+    }
+    __syncthreads();
+    const int T = sh.total;
+    int prefix = sh.warp_sums[warp] + incl - local;   // tiles before this thread's first sequence
+    if (T > 0) {
+        const long long g0 = span_begin(cta, T, G);
+        for (int b = b_lo; b < b_hi; ++b) {
+            const int nt = (clamp_len(lengths[b], Lmax) + tile_rows - 1) >> tile_shift;
+            if (nt > 0 && (long long)prefix <= g0 && g0 < (long long)prefix + nt) { sh.b0 = b; sh.p0 = prefix; }
+            prefix += nt;
+        }
+    }
+    __syncthreads();
+    return T;
+}
+
+// Walks the segments of one block's run.  All threads that use it hold identical state.
+struct SegmentWalker {
+    const int32_t* lengths;
+    int Lmax, tile_shift, B;
+    long long g0, g1;     // this block's run
+    long long g;          // next tile to hand out
+    int b, len, nt;       // current sequence
+    long long P;          // global index of its first tile
+
+    __host__ __device__ void init(const int32_t* lengths_, int B_, int Lmax_, int tile_shift_, int T, int G,
+                         int cta, int b0, int p0)
+    {
+        lengths = lengths_; B = B_; Lmax = Lmax_; tile_shift = tile_shift_;
+        g0 = span_begin(cta, T, G); g1 = span_begin(cta + 1, T, G); g = g0;
+        if (g0 < g1) {
+            b = b0; P = p0;
+            len = clamp_len(lengths[b], Lmax);
+            nt = (len + (1 << tile_shift) - 1) >> tile_shift;
+        }
+    }
+    __host__ __device__ bool done() const { return g >= g1; }
+    // Current segment: tiles [seg_t0, seg_t1) of sequence b (indices within the sequence).
+    __host__ __device__ int seg_t0() const { return (int)(g - P); }
+    __host__ __device__ int seg_t1() const { return (int)((g1 < P + nt ? g1 : P + nt) - P); }
+    __host__ __device__ bool seg_is_whole() const { return g == P && g1 >= P + nt; }
+    __host__ __device__ bool seg_owns_first_tile() const { return g == P; }
+    __host__ __device__ int seg_slot(int cta) const { return (P <= g0) ? 2 * cta : 2 * cta + 1; }
+    __host__ __device__ void next() {
+        g = (g1 < P + nt) ? g1 : P + nt;
+        if (g < g1) {
+            P += nt;
+            do {
+                ++b;
+                len = clamp_len(lengths[b], Lmax);
+                nt = (len + (1 << tile_shift) - 1) >> tile_shift;
+            } while (nt == 0 && b + 1 < B);
+        }
+    }
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Launchers (defined in their own translation units).
+cudaError_t launch_fma(const Params& p, cudaStream_t stream);
+cudaError_t launch_combine(const Params& p, cudaStream_t stream);
+cudaError_t launch_tc(const Params& p, cudaStream_t stream);
+bool tc_supported(int H, int D);
+
+}  // namespace mqa

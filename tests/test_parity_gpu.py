@@ -1,0 +1,150 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the
+same seeded inputs, element by element, within |err| <= 2e-3 * (1 + |ref|)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from mqa_workloads import WORKLOADS, make_custom, make_inputs, poison_padding
+from oracle import ref
+from paper_2211_05102_b200 import binding
+
+from gpu_util import assert_close, check, plans_for, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["tiny", "palm8b", "palm62b", "palm540b", "ragged32k"])
+def test_named_configs_full_size(name):
+    """The five configurations of the metric, at full size, under the heuristic's plan
+    (the launch configuration the benchmark times)."""
+    w = WORKLOADS[name]
+    q, k, v, lengths = make_inputs(w)
+    got = run_gpu(q, k, v, lengths, w.scale)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, w.scale)
+    worst = assert_close(got, expect, name)
+    print(f"{name}: max err/tol = {worst:.4f}")
+
+
+@pytest.mark.parametrize("name", ["tiny", "palm8b", "palm62b"])
+def test_named_configs_every_path(name):
+    w = WORKLOADS[name]
+    q, k, v, lengths = make_inputs(w)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, w.scale)
+    for plan in plans_for(w.B, w.H, w.D, w.Lmax, ctas=(None, 1, 7)):
+        got = run_gpu(q, k, v, lengths, w.scale, plan=plan)
+        assert_close(got, expect, f"{name} {plan}")
+
+
+EDGE_LENGTHS = [0, 1, 2, 3, 5, 17, 63, 64, 65, 127, 128, 129, 255, 256, 257, 300]
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("H", [1, 4, 16, 32, 48, 64])
+def test_edge_lengths(H, D):
+    B, Lmax = len(EDGE_LENGTHS), 300
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=1000 + H * 7 + D, lengths=EDGE_LENGTHS)
+    k, v = poison_padding(k, v, lengths, 0x7FC0)     # NaN beyond every length
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1.0 / math.sqrt(D))
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 1, 2, 3, 7, binding.MQA_MAX_CTAS)):
+        got = run_gpu(q, k, v, lengths, 1.0 / math.sqrt(D), plan=plan)
+        assert_close(got, expect, f"H={H} D={D} {plan}")
+        assert bool((got[0] == 0).all()), "length 0 must give an exactly zero row"
+
+
+@pytest.mark.parametrize("pattern", [0x7FC0, 0x7F80, 0xFF80])
+def test_padding_bits_never_reach_the_output(pattern):
+    B, H, D, Lmax = 6, 48, 256, 700
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=77, lengths=[700, 1, 129, 500, 64, 333])
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1 / 16)
+    k2, v2 = poison_padding(k, v, lengths, pattern)
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 5)):
+        assert_close(run_gpu(q, k2, v2, lengths, 1 / 16, plan=plan), expect, f"{plan}")
+
+
+def test_long_sequences_split_across_many_blocks():
+    B, H, D, Lmax = 3, 48, 256, 20000
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=78, lengths=[20000, 7, 12345])
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1 / 16)
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 1, 2, 3, 7, 148, binding.MQA_MAX_CTAS)):
+        assert_close(run_gpu(q, k, v, lengths, 1 / 16, plan=plan), expect, f"{plan}")
+
+
+def test_short_sequences_with_large_values():
+    """Lengths 2 and 3 with V scaled by 4: the case where a low-precision probability
+    would show (the output is a blend of very few large rows)."""
+    B, H, D, Lmax = 8, 48, 256, 8
+    q, k, v, _ = make_custom(B, H, D, Lmax, seed=79)
+    v = (v.float() * 4).to(torch.bfloat16)
+    lengths = torch.tensor([2, 3, 2, 3, 5, 2, 3, 8], dtype=torch.int32)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1 / 16)
+    for plan in plans_for(B, H, D, Lmax):
+        assert_close(run_gpu(q, k, v, lengths, 1 / 16, plan=plan), expect, f"{plan}")
+
+
+def test_all_equal_logits_give_the_mean():
+    B, H, D, Lmax = 2, 16, 128, 400
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=80, lengths=[400, 131])
+    q = torch.zeros_like(q)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 0.5)
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 3)):
+        assert_close(run_gpu(q, k, v, lengths, 0.5, plan=plan), expect, f"{plan}")
+
+
+@pytest.mark.parametrize("where", ["first", "middle", "last"])
+def test_one_dominant_logit(where):
+    B, H, D, Lmax = 2, 32, 256, 1000
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=81, lengths=[1000, 777])
+    for b in range(B):
+        n = int(lengths[b])
+        j = {"first": 0, "middle": n // 2, "last": n - 1}[where]
+        qm = q[b].float().mean(0)
+        k[b, j] = (qm * (400.0 / float(qm @ qm))).to(torch.bfloat16)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1 / 16)
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 1, 4)):
+        assert_close(run_gpu(q, k, v, lengths, 1 / 16, plan=plan), expect, f"{where} {plan}")
+
+
+def test_logits_that_keep_growing_along_the_sequence():
+    """The running maximum rises in every tile, so the accumulator is rescaled every time."""
+    B, H, D, Lmax = 2, 48, 256, 1500
+    q, k, v, lengths = make_custom(B, H, D, Lmax, seed=82, lengths=[1500, 901])
+    qm = q.float().mean(1)                                   # [B,D]
+    ramp = torch.arange(Lmax, dtype=torch.float32) / Lmax    # 0..1
+    for b in range(B):
+        k[b] = (k[b].float() * 0.05 + ramp[:, None] * qm[b][None, :] * (600.0 / float(qm[b] @ qm[b]))).to(torch.bfloat16)
+    expect = ref.mqa_decode_ref(q, k, v, lengths, 1 / 16)
+    for plan in plans_for(B, H, D, Lmax, ctas=(None, 1, 5)):
+        assert_close(run_gpu(q, k, v, lengths, 1 / 16, plan=plan), expect, f"{plan}")
+
+
+def test_same_plan_is_bit_identical_and_workspace_is_reusable():
+    w = WORKLOADS["palm8b"]
+    q, k, v, lengths = make_inputs(w)
+    ws = binding.alloc_workspace(w.B, w.H, w.D, w.Lmax)
+    a = run_gpu(q, k, v, lengths, w.scale, workspace=ws)
+    b = run_gpu(q, k, v, lengths, w.scale, workspace=ws)
+    assert torch.equal(a, b)
+    # a different problem through the same (larger) workspace, then the first again
+    q2, k2, v2, l2 = make_custom(3, w.H, w.D, 500, seed=83, lengths=[500, 0, 250])
+    ws_big = binding.alloc_workspace(w.B, w.H, w.D, w.Lmax)
+    expect2 = ref.mqa_decode_ref(q2, k2, v2, l2, w.scale)
+    run_gpu(q, k, v, lengths, w.scale, workspace=ws_big)
+    assert_close(run_gpu(q2, k2, v2, l2, w.scale, workspace=ws_big), expect2, "reuse")
+
+
+def test_host_entry_point_matches():
+    w = WORKLOADS["palm8b"]
+    q, k, v, lengths = make_inputs(w)
+    out = torch.empty((w.B, w.H, w.D), dtype=torch.float32).pin_memory()
+    scratch = torch.empty(binding.mqa_decode_host_scratch_bytes(w.B, w.H, w.D, w.Lmax), dtype=torch.uint8, device="cuda:0")
+    binding.mqa_decode_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), lengths.pin_memory(), out, w.scale, scratch)
+    assert_close(out, ref.mqa_decode_ref(q, k, v, lengths, w.scale), "host entry")
+
+
+def test_launch_count_is_reported():
+    w = WORKLOADS["tiny"]
+    q, k, v, lengths = make_inputs(w)
+    run_gpu(q, k, v, lengths, w.scale)
+    assert binding.mqa_last_launch_count() >= 1
