@@ -303,7 +303,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-sample-seqs", type=int, default=64,
+    ap.add_argument("--ref-sample-seqs", type=int, default=512,
                     help="sequences of the workload the CPU oracle is timed on")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
