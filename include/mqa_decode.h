@@ -171,6 +171,38 @@ int mqa_decode_host(const void* q_host, const void* k_cache_host, const void* v_
 int mqa_last_launch_count(void);
 
 /*
+ * Allocation-free variant of mqa_decode (the paper has no counterpart; this is
+ * a packaging convenience of this library).  It is for callers that cannot
+ * allocate device memory at all - code embedded in a host application that
+ * owns every byte of the GPU, a serving loop that may not enter the allocator,
+ * a sandbox where allocation calls are unavailable - and therefore cannot
+ * supply the workspace mqa_decode asks for.  The workspace is instead a fixed
+ * array of MQA_STATIC_WORKSPACE_BYTES inside the library's device image; every
+ * GPU that loads the library holds that much memory until the process exits.
+ *
+ * Arguments, layouts and results are those of mqa_decode, without the
+ * workspace.  Limits: the shape must fit the fixed array, i.e.
+ *   256 + roundup(8*B, 256) + 2 * 4*(2*roundup(H,4) + H*D) <= MQA_STATIC_WORKSPACE_BYTES;
+ * a larger shape returns MQA_ERR_WORKSPACE_TOO_SMALL and launches nothing.
+ * When the heuristic's block count would not fit, fewer blocks are used.
+ * The call makes no cudaMalloc/cudaFree and uses no allocating library
+ * routine.  The first call on each device looks up the array's device address
+ * (once per device, with that device current); make that first call outside of
+ * any stream capture.
+ *
+ * All calls on one device share the array, and it keeps the last call's
+ * contents: the call clears the part that must start at zero (the header) on
+ * `stream` before launching.  Calls whose kernels may overlap on the GPU
+ * (different streams without ordering) race on the array; order them.  A
+ * time-out of a bounded device-side wait cannot be read back through this
+ * entry point; use mqa_decode with mqa_check_status to diagnose one.
+ */
+#define MQA_STATIC_WORKSPACE_BYTES (20u << 20)
+int mqa_decode_static(const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* lengths, float* out,
+                      int B, int H, int D, int Lmax, float scale, void* stream);
+
+/*
  * Host replay of the device tile schedule, for tests and tooling (no device is
  * touched).  The K/V tiles of all sequences are numbered sequence-major and
  * block `cta` of `num_ctas` takes a contiguous run of them; each piece of a

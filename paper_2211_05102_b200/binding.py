@@ -31,7 +31,7 @@ MQA_MAX_CTAS = 592
 EXPORTS = [
     "mqa_status_string", "mqa_decode_workspace_bytes", "mqa_workspace_init", "mqa_decode_plan",
     "mqa_decode", "mqa_decode_with_plan", "mqa_decode_profiled", "mqa_check_status", "mqa_decode_host_scratch_bytes",
-    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule",
+    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static",
 ]
 
 
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_host_scratch_bytes.argtypes = [ci, ci, ci, ci]; L.mqa_decode_host_scratch_bytes.restype = sz
         L.mqa_decode_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, sz, vp]; L.mqa_decode_host.restype = ci
         L.mqa_last_launch_count.argtypes = []; L.mqa_last_launch_count.restype = ci
+        L.mqa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp]; L.mqa_decode_static.restype = ci
         L.mqa_debug_schedule.argtypes = [vp, ci, ci, ci, ci, ci, vp, ci]; L.mqa_debug_schedule.restype = ci
         _lib = L
     return _lib
@@ -165,6 +166,21 @@ def mqa_decode_profiled(q, k_cache, v_cache, lengths, out, scale: float, workspa
                                    ctypes.byref(plan) if plan is not None else None,
                                    workspace.data_ptr(), workspace.numel(), _stream_ptr(stream), handle)
     _check(rc, "mqa_decode_profiled")
+    return out
+
+
+MQA_STATIC_WORKSPACE_BYTES = 20 << 20
+
+
+def mqa_decode_static(q, k_cache, v_cache, lengths, out, scale: float, stream=None):
+    """mqa_decode for callers that cannot allocate device memory: no workspace argument,
+    the scratch is a fixed array inside the library (shapes beyond it are rejected)."""
+    B, H, D, Lmax = _shapes(q, k_cache, v_cache, lengths, out)
+    for t in (q, k_cache, v_cache, lengths, out):
+        assert t.is_cuda
+    rc = lib().mqa_decode_static(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), lengths.data_ptr(),
+                                 out.data_ptr(), B, H, D, Lmax, float(scale), _stream_ptr(stream))
+    _check(rc, "mqa_decode_static")
     return out
 
 
