@@ -9,7 +9,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmqa_decode.so")
 SOURCES = ["mqa_api.cu", "mqa_fma.cu", "mqa_combine.cu", "mqa_tc.cu", "mqa_static_ws.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC", "-lcuda"]
+              "-shared", "-Xcompiler", "-fPIC"]
 
 
 def _stale() -> bool:

@@ -1,6 +1,645 @@
-// tcgen05 tensor-core path (placeholder until the kernel lands).
+// Tensor-core multiquery decode kernel for sm_100a: TMA-staged K/V tiles, tcgen05
+// MMAs with accumulators in tensor memory, base-2 online softmax, partial writer.
+//
+// One persistent block per SM walks its run of 128-row K/V tiles (the flattened
+// schedule of mqa_common.cuh).  Each K/V tile is staged in shared memory ONCE by
+// TMA and used for all H query heads of its sequence - the multiquery saving of
+// the paper's Section 3.3.  Both products are issued "swapped" so that the long
+// axis sits on the 128 MMA rows and the heads on the narrow N side:
+//     S^T[l, h] = K_tile[l, :] . Q[h, :]          M = 128 rows, N = HP, K = D
+//     O^T[d, h] += V_tile^T[d, l] . P^T[l, h]     M = 128 (per 128-wide half of D), N = HP, K = 128
+// S^T lives in tensor memory with one cache row per lane, so a softmax thread owns
+// one cache row and all heads.  The probabilities go back through shared memory
+// as bf16 hi + lo halves (two MMAs), which keeps ~16 bits of each probability.
+//
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (and tensor-memory owner),
+// warps 4-7 = softmax + segment epilogue.  Every wait is bounded; when one runs
+// out the block records MQA_ERR_TIMEOUT in the workspace header and leaves.
 #include "mqa_common.cuh"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cudaTypedefs.h>
+
 namespace mqa {
-bool tc_supported(int, int) { return false; }
-cudaError_t launch_tc(const Params&, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kTcThreads = 256;
+constexpr int kTileShift = 7;
+constexpr int kTileRows = 128;
+constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 64 rows x 128 cols (V)
+constexpr int kMaxSlots = 12;
+constexpr int kMinSlots = 8;
+constexpr float kRescaleThreshold = 8.0f;  // base-2 logit units: rescale only when a logit exceeds m + 8
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds; only a deadlock gets here
+constexpr int kSoftmaxThreads = 128;
+constexpr int kSoftmaxWarp0 = 4;
+constexpr uint32_t kTmemCols = 256;        // S0 @0, S1 @64, O0 @128, O1 @192
+
+struct Barriers {
+    unsigned long long full[kMaxSlots];
+    unsigned long long empty[kMaxSlots];
+    unsigned long long q_full[2], q_empty[2];
+    unsigned long long s_full[2], s_empty[2];
+    unsigned long long p_full, p_empty;
+    unsigned long long o_full, o_empty;
+};
+
+struct Misc {
+    Barriers bars;
+    SchedShared sched;
+    uint32_t tmem_base;
+    int abort_flag;
+    float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
+};
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the block's abort flag) when the limit is hit
+// or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 63u) == 0u && (clock64() - t0 > kWaitLimitCycles || *abort_flag)) { *abort_flag = 1; return false; }
+    }
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, void* bar, int x, int y, int z, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate, issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on an mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(void* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float warp_max_f32(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// Barrier over the 128 softmax threads (named barrier 1) with an OR reduction of a flag.
+__device__ __forceinline__ bool softmax_bar_or(bool flag) {
+    uint32_t out, in = flag ? 1u : 0u;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"(in) : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle = 2 at bits 61..63).
+// K-major operand, rows of 128 B (64 bf16), 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// MN-major operand: 64 contiguous MN elements per row of 128 B, the next 64 MN elements
+// `mn_group_bytes` further on, 8-row K groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_mnmajor_sw128(uint32_t saddr, uint32_t mn_group_bytes) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_group_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; a_mn_major selects a transposed A.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
+
+// Position of one 128-row tile inside the block's run, shared by all roles.
+struct TileCursor {
+    SegmentWalker w;
+    int t, t1;        // current tile and end tile within the sequence
+    int seg;          // segment counter of this block
+    __device__ void init(const Params& p, int T, int cta, const SchedShared& sh) {
+        w.init(p.lengths, p.B, p.Lmax, kTileShift, T, p.num_ctas, cta, sh.b0, sh.p0);
+        seg = 0;
+        if (!w.done()) { t = w.seg_t0(); t1 = w.seg_t1(); }
+    }
+    __device__ bool valid() const { return !w.done(); }
+    __device__ bool first_in_seg() const { return t == w.seg_t0(); }
+    __device__ bool last_in_seg() const { return t + 1 == t1; }
+    __device__ int row0() const { return t << kTileShift; }
+    __device__ int nvalid() const { return min(kTileRows, w.len - row0()); }
+    __device__ void advance() {
+        if (++t == t1) {
+            w.next(); ++seg;
+            if (!w.done()) { t = w.seg_t0(); t1 = w.seg_t1(); }
+        }
+    }
+};
+
+// Ring bookkeeping: the producer and both consumers enumerate load items in the same order
+// K(0), K(1), V(0), K(2), V(1), ..., K(N-1), V(N-2), V(N-1); every item fills SPT consecutive slots.
+__device__ __forceinline__ int item_of_k(int n) { return n == 0 ? 0 : 2 * n - 1; }
+__device__ __forceinline__ int item_of_v(int n, int N) { return n == N - 1 ? 2 * N - 1 : 2 * n + 2; }
+
+template <int D, int HP>
+struct TcLayout {
+    static constexpr int SPT = D / 64;            // ring slots per K tile and per V tile
+    static constexpr int NACC = D / 128;          // 128-wide halves of D = output accumulators
+    static constexpr int kQBytes = HP * D * 2;    // one q buffer: D/64 chunks of [HP rows x 128 B]
+    static constexpr int kPBytes = HP * 128 * 2;  // one probability buffer: 2 chunks of [HP rows x 128 B]
+    static constexpr int kFixed = 2 * kQBytes + 2 * kPBytes + (int)sizeof(Misc);
+    static int slots_for(int smem_limit) {
+        int n = (smem_limit - 1024 - kFixed) / kSlotBytes;
+        return n > kMaxSlots ? kMaxSlots : n;
+    }
+    static int smem_bytes(int nslots) { return 1024 + nslots * kSlotBytes + kFixed; }
+};
+
+template <int D, int HP>
+__global__ void __launch_bounds__(kTcThreads, 1)
+mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+              const __grid_constant__ CUtensorMap map_v, const int nslots)
+{
+    using L = TcLayout<D, HP>;
+    constexpr int SPT = L::SPT, NACC = L::NACC;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* ring = smem;
+    unsigned char* q_buf = ring + (size_t)nslots * kSlotBytes;       // 2 buffers
+    unsigned char* p_hi = q_buf + 2 * L::kQBytes;
+    unsigned char* p_lo = p_hi + L::kPBytes;
+    Misc& misc = *reinterpret_cast<Misc*>(p_lo + L::kPBytes);
+    Barriers& bars = misc.bars;
+    volatile int* abort_flag = &misc.abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x, G = p.num_ctas, H = p.H;
+
+    if (tid == 0) {
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars.q_full[i], 1); mbar_init(&bars.q_empty[i], 1);
+            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], kSoftmaxThreads);
+        }
+        mbar_init(&bars.p_full, kSoftmaxThreads); mbar_init(&bars.p_empty, 1);
+        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, kSoftmaxThreads);
+        misc.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) {   // tensor-memory allocation (one warp owns it for the whole kernel)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tc_fence_before();
+    }
+    const int T = schedule_prologue<kTcThreads>(p.lengths, p.B, p.Lmax, kTileShift, G, cta, misc.sched);   // has __syncthreads
+    tc_fence_after();
+    const uint32_t tmem = misc.tmem_base;
+    if (cta == 0 && tid == 0) {
+        ws_header(p.workspace)[kHdrTotalTiles] = T;
+        ws_header(p.workspace)[kHdrNumCtas] = G;
+    }
+    const int N = (T > 0) ? (int)(span_begin(cta + 1, T, G) - span_begin(cta, T, G)) : 0;   // tiles of this block
+
+    if (N > 0) {
+        if (warp == 0 && lane == 0) {
+            // =============================== TMA producer ===============================
+            uint64_t policy;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+            uint64_t policy_q;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy_q));
+            TileCursor ck, cv;
+            ck.init(p, T, cta, misc.sched);
+            cv = ck;
+            int slot_seq = 0;          // running slot counter = item * SPT + chunk
+            bool ok = true;
+            auto acquire = [&](int s) -> unsigned char* {
+                const int slot = s % nslots, use = s / nslots;
+                if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return nullptr; }
+                mbar_expect_tx(&bars.full[slot], kSlotBytes);
+                return ring + (size_t)slot * kSlotBytes;
+            };
+            auto load_k = [&](const TileCursor& c) {
+                if (c.first_in_seg()) {   // stage this sequence's queries first
+                    const int qb = c.seg & 1;
+                    if (!mbar_wait(&bars.q_empty[qb], ((c.seg >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                    mbar_expect_tx(&bars.q_full[qb], L::kQBytes);
+                    for (int ch = 0; ch < SPT; ++ch)
+                        tma_load_3d(q_buf + qb * L::kQBytes + ch * (HP * 128), &map_q, &bars.q_full[qb], ch * 64, 0, c.w.b, policy_q);
+                }
+                for (int ch = 0; ch < SPT && ok; ++ch) {
+                    unsigned char* dst = acquire(slot_seq);
+                    if (!dst) return;
+                    tma_load_3d(dst, &map_k, &bars.full[slot_seq % nslots], ch * 64, c.row0(), c.w.b, policy);
+                    ++slot_seq;
+                }
+            };
+            auto load_v = [&](const TileCursor& c) {
+                for (int vi = 0; vi < SPT && ok; ++vi) {
+                    const int r = vi / NACC, j = vi % NACC;
+                    unsigned char* dst = acquire(slot_seq);
+                    if (!dst) return;
+                    void* bar = &bars.full[slot_seq % nslots];
+                    tma_load_3d(dst, &map_v, bar, j * 128, c.row0() + r * 64, c.w.b, policy);
+                    tma_load_3d(dst + 8192, &map_v, bar, j * 128 + 64, c.row0() + r * 64, c.w.b, policy);
+                    ++slot_seq;
+                }
+            };
+            load_k(ck); ck.advance();
+            while (ok && cv.valid()) {
+                if (ck.valid()) { load_k(ck); ck.advance(); }
+                if (ok) { load_v(cv); cv.advance(); }
+            }
+            if (!ok) {
+                // give copies already in flight a bounded chance to land before the block retires
+                for (int s = max(0, slot_seq - nslots); s < slot_seq; ++s) {
+                    const int slot = s % nslots, use = s / nslots;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&bars.full[slot], use & 1) && clock64() - t0 < kWaitLimitCycles) {}
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // =============================== MMA issuer ===============================
+            constexpr uint32_t idesc_qk = make_idesc(HP, false);
+            constexpr uint32_t idesc_pv = make_idesc(HP, true);
+            TileCursor ck, cv;
+            ck.init(p, T, cta, misc.sched);
+            cv = ck;
+            int nq = 0, np = 0;
+            bool ok = true;
+            auto issue_qk = [&](const TileCursor& c) {
+                const int sb = nq & 1;
+                if (!mbar_wait(&bars.s_empty[sb], ((nq >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                const int qb = c.seg & 1;
+                if (c.first_in_seg() && !mbar_wait(&bars.q_full[qb], (c.seg >> 1) & 1, abort_flag)) { ok = false; return; }
+                const uint32_t d_tmem = tmem + (uint32_t)(sb * 64);
+                const int s0 = item_of_k(nq) * SPT;
+                for (int ch = 0; ch < SPT; ++ch) {
+                    const int s = s0 + ch, slot = s % nslots, use = s / nslots;
+                    if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                    tc_fence_after();
+                    const uint64_t da = desc_kmajor_sw128(smem_u32(ring + (size_t)slot * kSlotBytes));
+                    const uint64_t db = desc_kmajor_sw128(smem_u32(q_buf + qb * L::kQBytes + ch * (HP * 128)));
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
+                        umma_bf16(d_tmem, da + (uint64_t)(ks * 2), db + (uint64_t)(ks * 2), idesc_qk, (ch | ks) ? 1u : 0u);
+                    umma_commit(&bars.empty[slot]);
+                }
+                umma_commit(&bars.s_full[sb]);
+                if (c.last_in_seg()) umma_commit(&bars.q_empty[qb]);
+                ++nq;
+            };
+            auto issue_pv = [&](const TileCursor& c) {
+                if (!mbar_wait(&bars.p_full, np & 1, abort_flag)) { ok = false; return; }
+                if (c.first_in_seg() && !mbar_wait(&bars.o_empty, (c.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
+                tc_fence_after();
+                const int s0 = item_of_v(np, N) * SPT;
+                for (int vi = 0; vi < SPT; ++vi) {
+                    const int r = vi / NACC, j = vi % NACC;
+                    const int s = s0 + vi, slot = s % nslots, use = s / nslots;
+                    if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem + 128u + (uint32_t)(j * 64);
+                    const uint64_t da = desc_mnmajor_sw128(smem_u32(ring + (size_t)slot * kSlotBytes), 8192);
+                    const uint64_t dbh = desc_kmajor_sw128(smem_u32(p_hi + r * (HP * 128)));
+                    const uint64_t dbl = desc_kmajor_sw128(smem_u32(p_lo + r * (HP * 128)));
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {   // 4 x 16 cache rows per 64-row slot
+                        const uint32_t acc = (c.first_in_seg() && r == 0 && ks == 0) ? 0u : 1u;
+                        umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbh + (uint64_t)(ks * 2), idesc_pv, acc);
+                        umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbl + (uint64_t)(ks * 2), idesc_pv, 1u);
+                    }
+                    umma_commit(&bars.empty[slot]);
+                }
+                umma_commit(&bars.p_empty);
+                if (c.last_in_seg()) umma_commit(&bars.o_full);
+                ++np;
+            };
+            issue_qk(ck); ck.advance();
+            while (ok && cv.valid()) {
+                if (ck.valid()) { issue_qk(ck); ck.advance(); }
+                if (ok) { issue_pv(cv); cv.advance(); }
+            }
+        } else if (warp >= kSoftmaxWarp0) {
+            // =============================== softmax + epilogue ===============================
+            const int row = tid - kSoftmaxWarp0 * 32;          // cache row within the tile = tensor-memory lane
+            const int wq = warp - kSoftmaxWarp0;               // lane quadrant of this warp
+            const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
+            TileCursor c;
+            c.init(p, T, cta, misc.sched);
+            int ns = 0;
+            bool ok = true;
+            float m[HP], l[HP];
+            while (ok && c.valid()) {
+                // ---------------- new segment ----------------
+                const int b = c.w.b, seg = c.seg;
+                const bool whole = c.w.seg_is_whole();
+                const int slot_id = c.w.seg_slot(cta);
+                if (c.w.seg_owns_first_tile() && row == 0) {
+                    SeqInfo si;
+                    si.first_slot = whole ? -1 : slot_id;
+                    si.last_cta = cta_of_tile(c.w.P + c.w.nt - 1, T, G);
+                    ws_seqinfo(p.workspace)[b] = si;
+                }
+#pragma unroll
+                for (int h = 0; h < HP; ++h) { m[h] = -INFINITY; l[h] = 0.f; }
+                bool first = true;
+                for (;;) {
+                    const int sb = ns & 1;
+                    const int nvalid = c.nvalid();
+                    const bool last = c.last_in_seg();
+                    if (!mbar_wait(&bars.s_full[sb], (ns >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    float y[HP];
+#pragma unroll
+                    for (int h0 = 0; h0 < HP; h0 += 16) tmem_ld16(lane_base + (uint32_t)(sb * 64 + h0), &y[h0]);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(&bars.s_empty[sb]);
+                    const bool valid = row < nvalid;
+                    bool exceed = false;
+#pragma unroll
+                    for (int h = 0; h < HP; ++h) {
+                        y[h] = valid ? y[h] * p.scale_log2 : -INFINITY;
+                        exceed |= (y[h] > m[h] + kRescaleThreshold);
+                    }
+                    const bool need = softmax_bar_or(exceed);
+                    // probabilities of tile ns overwrite the buffer read by the MMAs of tile ns-1
+                    if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (need) {
+                        // exact per-head maximum of this tile, then move the reference m up
+#pragma unroll
+                        for (int h = 0; h < HP; ++h) {
+                            const float wm = warp_max_f32(y[h]);
+                            if (lane == (h & 31)) misc.wred[wq][h] = wm;
+                        }
+                        softmax_bar_sync();
+                        float alpha[HP];
+#pragma unroll
+                        for (int h = 0; h < HP; ++h) {
+                            const float tm = fmaxf(fmaxf(misc.wred[0][h], misc.wred[1][h]), fmaxf(misc.wred[2][h], misc.wred[3][h]));
+                            const float m_new = fmaxf(m[h], tm);
+                            alpha[h] = (m[h] == -INFINITY) ? 0.f : exp2f(m[h] - m_new);
+                            l[h] *= alpha[h];
+                            m[h] = m_new;
+                        }
+                        softmax_bar_sync();   // wred may be reused by the next tile
+                        if (!first) {
+                            // rescale the accumulators in tensor memory (their MMAs have completed: p_empty)
+                            tc_fence_after();
+#pragma unroll
+                            for (int j = 0; j < NACC; ++j) {
+#pragma unroll
+                                for (int h0 = 0; h0 < HP; h0 += 16) {
+                                    float o[16];
+                                    const uint32_t ta = lane_base + 128u + (uint32_t)(j * 64 + h0);
+                                    tmem_ld16(ta, o);
+                                    tmem_wait_ld();
+#pragma unroll
+                                    for (int i = 0; i < 16; ++i) o[i] *= alpha[h0 + i];
+                                    tmem_st16(ta, o);
+                                }
+                            }
+                            tmem_wait_st();
+                            tc_fence_before();
+                        }
+                    }
+                    // p = 2^(y - m); write bf16 hi and lo parts into the K-major, 128B-swizzled B operand
+                    {
+                        const int chunk = row >> 6, col = row & 63;
+                        const uint32_t unit = (uint32_t)(col >> 3), within = (uint32_t)(col & 7) * 2u;
+                        unsigned char* ph = p_hi + chunk * (HP * 128);
+                        unsigned char* pl = p_lo + chunk * (HP * 128);
+#pragma unroll
+                        for (int h = 0; h < HP; ++h) {
+                            const float pr = exp2f(y[h] - m[h]);          // 0 for masked rows (y = -inf, m finite)
+                            l[h] += pr;
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(pr);
+                            const __nv_bfloat16 lo = __float2bfloat16_rn(pr - __bfloat162float(hi));
+                            const uint32_t off = (uint32_t)h * 128u + ((unit ^ (uint32_t)(h & 7)) << 4) + within;
+                            *reinterpret_cast<__nv_bfloat16*>(ph + off) = hi;
+                            *reinterpret_cast<__nv_bfloat16*>(pl + off) = lo;
+                        }
+                    }
+                    if (nvalid < kTileRows) {
+                        // rows beyond the sequence may hold any bits: zero them in the staged V tile
+                        const int s0 = item_of_v(ns, N) * SPT;
+                        for (int vi = 0; vi < SPT; ++vi) {
+                            const int r = vi / NACC;
+                            const int s = s0 + vi, slot = s % nslots, use = s / nslots;
+                            if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; break; }
+                            if (!valid && (row >> 6) == r) {
+                                uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (row & 63) * 128);
+                                uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + (row & 63) * 128);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) { dst0[i] = make_uint4(0, 0, 0, 0); dst1[i] = make_uint4(0, 0, 0, 0); }
+                            }
+                        }
+                        if (!ok) break;
+                    }
+                    fence_proxy_async();
+                    mbar_arrive(&bars.p_full);
+                    first = false;
+                    ++ns;
+                    c.advance();
+                    if (last) break;
+                }
+                if (!ok) break;
+                // ---------------- segment epilogue ----------------
+                // row sums over the 128 cache-row lanes
+#pragma unroll
+                for (int h = 0; h < HP; ++h) {
+                    float v = l[h];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane == (h & 31)) misc.wred[wq][h] = v;
+                }
+                softmax_bar_sync();
+                float lsum[HP];
+#pragma unroll
+                for (int h = 0; h < HP; ++h) lsum[h] = (misc.wred[0][h] + misc.wred[1][h]) + (misc.wred[2][h] + misc.wred[3][h]);
+                float oscale[HP];   // 1/l for a direct write, 1 for an unnormalised partial
+#pragma unroll
+                for (int h = 0; h < HP; ++h) oscale[h] = whole ? 1.f / lsum[h] : 1.f;
+                softmax_bar_sync();
+                if (!mbar_wait(&bars.o_full, seg & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, slot_id);
+                const int Hp4 = round_up(H, 4);
+                if (!whole && row < H) {
+                    // m is identical in every thread; thread `row` stores head `row`
+                    float mv = 0.f, lv = 0.f;
+#pragma unroll
+                    for (int h = 0; h < HP; ++h) if (h == row) { mv = m[h]; lv = lsum[h]; }
+                    slot_ptr[row] = mv;
+                    slot_ptr[Hp4 + row] = lv;
+                }
+#pragma unroll
+                for (int j = 0; j < NACC; ++j) {
+                    const int d = j * 128 + row;
+#pragma unroll
+                    for (int h0 = 0; h0 < HP; h0 += 16) {
+                        float o[16];
+                        tmem_ld16(lane_base + 128u + (uint32_t)(j * 64 + h0), o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int h = h0 + i;
+                            if (h < H) {
+                                if (whole) p.out[((size_t)b * H + h) * D + d] = o[i] * oscale[h];
+                                else slot_ptr[2 * Hp4 + (size_t)h * D + d] = o[i];
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(&bars.o_empty);
+            }
+        }
+    }
+
+    __syncwarp();
+    __syncthreads();
+    if (tid == 0 && misc.abort_flag) atomicExch(ws_header(p.workspace) + kHdrStatus, 7 /* MQA_ERR_TIMEOUT */);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn()
+{
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = []() -> PFN_cuTensorMapEncodeTiled_v12000 {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }();
+    return fn;
+}
+
+// 3-D bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box [1][box1][64], 128-byte swizzle, zero fill.
+bool encode_map(CUtensorMap* map, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box1)
+{
+    auto fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {dim0, dim1, dim2};
+    cuuint64_t strides[2] = {dim0 * 2, dim0 * dim1 * 2};
+    cuuint32_t box[3] = {64, box1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int HP>
+cudaError_t launch_tc_t(const Params& p, cudaStream_t stream)
+{
+    using L = TcLayout<D, HP>;
+    int dev = 0, smem_limit = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    const int nslots = L::slots_for(smem_limit);
+    if (nslots < kMinSlots) return cudaErrorInvalidConfiguration;
+    const int smem = L::smem_bytes(nslots);
+    CUtensorMap mq, mk, mv;
+    if (!encode_map(&mq, p.q, p.D, p.H, p.B, HP) || !encode_map(&mk, p.k, p.D, p.Lmax, p.B, 128) ||
+        !encode_map(&mv, p.v, p.D, p.Lmax, p.B, 64))
+        return cudaErrorInvalidValue;
+    e = cudaFuncSetAttribute(mqa_tc_kernel<D, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    mqa_tc_kernel<D, HP><<<p.num_ctas, kTcThreads, smem, stream>>>(p, mq, mk, mv, nslots);
+    return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_tc_d(const Params& p, cudaStream_t stream)
+{
+    const int hp = round_up(p.H, 16);
+    switch (hp) {
+        case 16: return launch_tc_t<D, 16>(p, stream);
+        case 32: return launch_tc_t<D, 32>(p, stream);
+        case 48: return launch_tc_t<D, 48>(p, stream);
+        case 64: return launch_tc_t<D, 64>(p, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+bool tc_supported(int H, int D) { return (D == 128 || D == 256) && H >= 8 && H <= kMaxHeads; }
+
+cudaError_t launch_tc(const Params& p, cudaStream_t stream)
+{
+    if (p.tile_shift != kTileShift) return cudaErrorInvalidValue;
+    switch (p.D) {
+        case 128: return launch_tc_d<128>(p, stream);
+        case 256: return launch_tc_d<256>(p, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace mqa
