@@ -129,6 +129,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = tile_shift_of(plan->tile_rows);
     p.num_ctas = plan->num_ctas;
+    p.lo_max_len = 0x7fffffff;
     p.workspace = static_cast<unsigned char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 

@@ -55,6 +55,7 @@ struct Params {
     float scale_log2;         // scale * log2(e): logits are kept in the base-2 domain
     int tile_shift;           // log2(tile_rows)
     int num_ctas;             // G
+    int lo_max_len;           // tensor-core path: sequences up to this length use hi+lo bf16 probabilities
     unsigned char* workspace;
 };
 

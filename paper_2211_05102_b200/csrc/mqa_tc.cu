@@ -21,11 +21,13 @@
 #include <cuda_bf16.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
+
 namespace mqa {
 
 namespace {
 
-constexpr int kTcThreads = 256;
+constexpr int kHeadsPerThread = 16;        // a softmax thread owns one cache row and 16 heads
 constexpr int kTileShift = 7;
 constexpr int kTileRows = 128;
 constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 64 rows x 128 cols (V)
@@ -33,7 +35,6 @@ constexpr int kMaxSlots = 12;
 constexpr int kMinSlots = 8;
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logit units: rescale only when a logit exceeds m + 8
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds; only a deadlock gets here
-constexpr int kSoftmaxThreads = 128;
 constexpr int kSoftmaxWarp0 = 4;
 constexpr uint32_t kTmemCols = 256;        // S0 @0, S1 @64, O0 @128, O1 @192
 
@@ -52,7 +53,26 @@ struct Misc {
     uint32_t tmem_base;
     int abort_flag;
     float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
+    __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
+    __align__(16) float alpha[kMaxHeads];  // rescale factors; row sums in the epilogue
 };
+
+// Optional cycle accounting (compile with -DMQA_TC_PROFILE): block 0 adds the cycles each role
+// spends in each wait to workspace header words 16.., read back by tuning scripts.
+#ifdef MQA_TC_PROFILE
+#define PROF_BEGIN() const long long prof_t0_ = clock64()
+#ifndef MQA_PROF_BLOCK
+#define MQA_PROF_BLOCK 0
+#endif
+#define PROF_END(idx) do { if (blockIdx.x == MQA_PROF_BLOCK && (threadIdx.x == 0 || threadIdx.x == 32 || threadIdx.x == 128)) \
+    atomicAdd(ws_header(p.workspace) + 16 + (idx), (int)(clock64() - prof_t0_)); } while (0)
+#else
+#define PROF_BEGIN() do {} while (0)
+#define PROF_END(idx) do {} while (0)
+#endif
+enum { kProfProdEmpty = 0, kProfMmaSEmpty, kProfMmaQFull, kProfMmaKFull, kProfMmaPFull, kProfMmaOEmpty, kProfMmaVFull,
+       kProfSmSFull, kProfSmBar, kProfSmPEmpty, kProfSmRescale, kProfSmStore, kProfSmEpilogue, kProfSmTotal, kProfMmaTotal,
+       kProfProdTotal, kProfSmLoad, kProfSmOFull };
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -135,23 +155,38 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ float ex2_approx(float x) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one_sync() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+        "elect.sync rx|px, 0xffffffff;\n\t"
+        "@px mov.s32 %0, 1;\n\t}"
+        : "+r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ float warp_max_f32(float v) {
     float r;
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-// Barrier over the 128 softmax threads (named barrier 1) with an OR reduction of a flag.
-__device__ __forceinline__ bool softmax_bar_or(bool flag) {
+// Barrier over the softmax threads (named barrier 1) with an OR reduction of a flag.
+__device__ __forceinline__ bool softmax_bar_or(bool flag, int nthreads) {
     uint32_t out, in = flag ? 1u : 0u;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, 128, p;\n\t"
+        "bar.red.or.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(out) : "r"(in) : "memory");
+        : "=r"(out) : "r"(in), "r"(nthreads) : "memory");
     return out != 0;
 }
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void softmax_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 // Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle = 2 at bits 61..63).
 // K-major operand, rows of 128 B (64 bf16), 8-row groups 1024 B apart.
@@ -165,10 +200,10 @@ __device__ __forceinline__ uint64_t desc_mnmajor_sw128(uint32_t saddr, uint32_t 
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_group_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; a_mn_major selects a transposed A.
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; *_mn_major selects a transposed operand.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
 // Position of one 128-row tile inside the block's run, shared by all roles.
@@ -201,10 +236,13 @@ __device__ __forceinline__ int item_of_v(int n, int N) { return n == N - 1 ? 2 *
 
 template <int D, int HP>
 struct TcLayout {
+    static constexpr int HG = HP / kHeadsPerThread;          // head groups = softmax warpgroups
+    static constexpr int kSoftmaxThreads = 128 * HG;
+    static constexpr int kThreads = 128 + kSoftmaxThreads;   // warps 0-3: producer, MMA issuer, two idle
     static constexpr int SPT = D / 64;            // ring slots per K tile and per V tile
     static constexpr int NACC = D / 128;          // 128-wide halves of D = output accumulators
     static constexpr int kQBytes = HP * D * 2;    // one q buffer: D/64 chunks of [HP rows x 128 B]
-    static constexpr int kPBytes = HP * 128 * 2;  // one probability buffer: 2 chunks of [HP rows x 128 B]
+    static constexpr int kPBytes = 128 * 128;     // one probability buffer: 128 cache rows x 128 B (up to 64 heads)
     static constexpr int kFixed = 2 * kQBytes + 2 * kPBytes + (int)sizeof(Misc);
     static int slots_for(int smem_limit) {
         int n = (smem_limit - 1024 - kFixed) / kSlotBytes;
@@ -214,7 +252,7 @@ struct TcLayout {
 };
 
 template <int D, int HP>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(TcLayout<D, HP>::kThreads, 1)
 mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, const int nslots)
 {
@@ -230,17 +268,22 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     Barriers& bars = misc.bars;
     volatile int* abort_flag = &misc.abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform in the compiler's eyes
+#ifdef MQA_TC_PROFILE
+    unsigned long long prof_ns0 = 0; long long prof_c0 = 0;
+    if (tid == 0) { asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_ns0)); prof_c0 = clock64(); }
+#endif
     const int cta = blockIdx.x, G = p.num_ctas, H = p.H;
 
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars.q_full[i], 1); mbar_init(&bars.q_empty[i], 1);
-            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], kSoftmaxThreads);
+            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads);
         }
-        mbar_init(&bars.p_full, kSoftmaxThreads); mbar_init(&bars.p_empty, 1);
-        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, kSoftmaxThreads);
+        mbar_init(&bars.p_full, L::kSoftmaxThreads); mbar_init(&bars.p_empty, 1);
+        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, L::kSoftmaxThreads);
         misc.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
@@ -250,7 +293,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         tc_fence_before();
     }
-    const int T = schedule_prologue<kTcThreads>(p.lengths, p.B, p.Lmax, kTileShift, G, cta, misc.sched);   // has __syncthreads
+    const int T = schedule_prologue<L::kThreads>(p.lengths, p.B, p.Lmax, kTileShift, G, cta, misc.sched);   // has __syncthreads
     tc_fence_after();
     const uint32_t tmem = misc.tmem_base;
     if (cta == 0 && tid == 0) {
@@ -260,46 +303,59 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     const int N = (T > 0) ? (int)(span_begin(cta + 1, T, G) - span_begin(cta, T, G)) : 0;   // tiles of this block
 
     if (N > 0) {
-        if (warp == 0 && lane == 0) {
-            // =============================== TMA producer ===============================
-            uint64_t policy;
+        if (warp == 0) {
+            // =============================== TMA producer (whole warp waits, one lane issues) ===============================
+            uint64_t policy, policy_q;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-            uint64_t policy_q;
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy_q));
             TileCursor ck, cv;
             ck.init(p, T, cta, misc.sched);
             cv = ck;
             int slot_seq = 0;          // running slot counter = item * SPT + chunk
             bool ok = true;
-            auto acquire = [&](int s) -> unsigned char* {
-                const int slot = s % nslots, use = s / nslots;
-                if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return nullptr; }
-                mbar_expect_tx(&bars.full[slot], kSlotBytes);
-                return ring + (size_t)slot * kSlotBytes;
-            };
+            PROF_BEGIN();
             auto load_k = [&](const TileCursor& c) {
                 if (c.first_in_seg()) {   // stage this sequence's queries first
                     const int qb = c.seg & 1;
                     if (!mbar_wait(&bars.q_empty[qb], ((c.seg >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
-                    mbar_expect_tx(&bars.q_full[qb], L::kQBytes);
-                    for (int ch = 0; ch < SPT; ++ch)
-                        tma_load_3d(q_buf + qb * L::kQBytes + ch * (HP * 128), &map_q, &bars.q_full[qb], ch * 64, 0, c.w.b, policy_q);
+                    if (elect_one_sync()) {
+                        mbar_expect_tx(&bars.q_full[qb], L::kQBytes);
+                        for (int ch = 0; ch < SPT; ++ch)
+                            tma_load_3d(q_buf + qb * L::kQBytes + ch * (HP * 128), &map_q, &bars.q_full[qb], ch * 64, 0, c.w.b, policy_q);
+                    }
+                    __syncwarp();
                 }
-                for (int ch = 0; ch < SPT && ok; ++ch) {
-                    unsigned char* dst = acquire(slot_seq);
-                    if (!dst) return;
-                    tma_load_3d(dst, &map_k, &bars.full[slot_seq % nslots], ch * 64, c.row0(), c.w.b, policy);
+                for (int ch = 0; ch < SPT; ++ch) {
+                    const int slot = slot_seq % nslots, use = slot_seq / nslots;
+                    {
+                        PROF_BEGIN();
+                        if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return; }
+                        PROF_END(kProfProdEmpty);
+                    }
+                    if (elect_one_sync()) {
+                        mbar_expect_tx(&bars.full[slot], kSlotBytes);
+                        tma_load_3d(ring + (size_t)slot * kSlotBytes, &map_k, &bars.full[slot], ch * 64, c.row0(), c.w.b, policy);
+                    }
+                    __syncwarp();
                     ++slot_seq;
                 }
             };
             auto load_v = [&](const TileCursor& c) {
-                for (int vi = 0; vi < SPT && ok; ++vi) {
+                for (int vi = 0; vi < SPT; ++vi) {
                     const int r = vi / NACC, j = vi % NACC;
-                    unsigned char* dst = acquire(slot_seq);
-                    if (!dst) return;
-                    void* bar = &bars.full[slot_seq % nslots];
-                    tma_load_3d(dst, &map_v, bar, j * 128, c.row0() + r * 64, c.w.b, policy);
-                    tma_load_3d(dst + 8192, &map_v, bar, j * 128 + 64, c.row0() + r * 64, c.w.b, policy);
+                    const int slot = slot_seq % nslots, use = slot_seq / nslots;
+                    {
+                        PROF_BEGIN();
+                        if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return; }
+                        PROF_END(kProfProdEmpty);
+                    }
+                    if (elect_one_sync()) {
+                        unsigned char* dst = ring + (size_t)slot * kSlotBytes;
+                        mbar_expect_tx(&bars.full[slot], kSlotBytes);
+                        tma_load_3d(dst, &map_v, &bars.full[slot], j * 128, c.row0() + r * 64, c.w.b, policy);
+                        tma_load_3d(dst + 8192, &map_v, &bars.full[slot], j * 128 + 64, c.row0() + r * 64, c.w.b, policy);
+                    }
+                    __syncwarp();
                     ++slot_seq;
                 }
             };
@@ -308,6 +364,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 if (ck.valid()) { load_k(ck); ck.advance(); }
                 if (ok) { load_v(cv); cv.advance(); }
             }
+            PROF_END(kProfProdTotal);
             if (!ok) {
                 // give copies already in flight a bounded chance to land before the block retires
                 for (int s = max(0, slot_seq - nslots); s < slot_seq; ++s) {
@@ -316,167 +373,243 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     while (!mbar_try_wait(&bars.full[slot], use & 1) && clock64() - t0 < kWaitLimitCycles) {}
                 }
             }
-        } else if (warp == 1 && lane == 0) {
-            // =============================== MMA issuer ===============================
-            constexpr uint32_t idesc_qk = make_idesc(HP, false);
-            constexpr uint32_t idesc_pv = make_idesc(HP, true);
+        } else if (warp == 1) {
+            // =============================== MMA issuer (whole warp waits, one lane issues) ===============================
+            constexpr uint32_t idesc_qk = make_idesc(HP, false, false);
+            constexpr uint32_t idesc_pv = make_idesc(HP, true, true);
             TileCursor ck, cv;
             ck.init(p, T, cta, misc.sched);
             cv = ck;
             int nq = 0, np = 0;
             bool ok = true;
+            const uint32_t ring_addr = smem_u32(ring), q_addr = smem_u32(q_buf);
+            const uint32_t phi_addr = smem_u32(p_hi), plo_addr = smem_u32(p_lo);
+            PROF_BEGIN();
             auto issue_qk = [&](const TileCursor& c) {
                 const int sb = nq & 1;
-                if (!mbar_wait(&bars.s_empty[sb], ((nq >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                { PROF_BEGIN();
+                  if (!mbar_wait(&bars.s_empty[sb], ((nq >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                  PROF_END(kProfMmaSEmpty); }
                 const int qb = c.seg & 1;
-                if (c.first_in_seg() && !mbar_wait(&bars.q_full[qb], (c.seg >> 1) & 1, abort_flag)) { ok = false; return; }
+                if (c.first_in_seg()) {
+                    PROF_BEGIN();
+                    if (!mbar_wait(&bars.q_full[qb], (c.seg >> 1) & 1, abort_flag)) { ok = false; return; }
+                    PROF_END(kProfMmaQFull);
+                }
                 const uint32_t d_tmem = tmem + (uint32_t)(sb * 64);
                 const int s0 = item_of_k(nq) * SPT;
                 for (int ch = 0; ch < SPT; ++ch) {
                     const int s = s0 + ch, slot = s % nslots, use = s / nslots;
-                    if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                    { PROF_BEGIN();
+                      if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                      PROF_END(kProfMmaKFull); }
                     tc_fence_after();
-                    const uint64_t da = desc_kmajor_sw128(smem_u32(ring + (size_t)slot * kSlotBytes));
-                    const uint64_t db = desc_kmajor_sw128(smem_u32(q_buf + qb * L::kQBytes + ch * (HP * 128)));
+                    const uint64_t da = desc_kmajor_sw128(ring_addr + (uint32_t)slot * kSlotBytes);
+                    const uint64_t db = desc_kmajor_sw128(q_addr + (uint32_t)(qb * L::kQBytes + ch * (HP * 128)));
+                    if (elect_one_sync()) {
+#ifndef MQA_X_SKIP_QK
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
-                        umma_bf16(d_tmem, da + (uint64_t)(ks * 2), db + (uint64_t)(ks * 2), idesc_qk, (ch | ks) ? 1u : 0u);
-                    umma_commit(&bars.empty[slot]);
+                        for (int ks = 0; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
+                            umma_bf16(d_tmem, da + (uint64_t)(ks * 2), db + (uint64_t)(ks * 2), idesc_qk, (ch | ks) ? 1u : 0u);
+#endif
+                        umma_commit(&bars.empty[slot]);
+                        if (ch == SPT - 1) {
+                            umma_commit(&bars.s_full[sb]);
+                            if (c.last_in_seg()) umma_commit(&bars.q_empty[qb]);
+                        }
+                    }
+                    __syncwarp();
                 }
-                umma_commit(&bars.s_full[sb]);
-                if (c.last_in_seg()) umma_commit(&bars.q_empty[qb]);
                 ++nq;
             };
-            auto issue_pv = [&](const TileCursor& c) {
-                if (!mbar_wait(&bars.p_full, np & 1, abort_flag)) { ok = false; return; }
-                if (c.first_in_seg() && !mbar_wait(&bars.o_empty, (c.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
+            auto issue_pv = [&](const TileCursor& c, bool use_lo) {
+                { PROF_BEGIN();
+                  if (!mbar_wait(&bars.p_full, np & 1, abort_flag)) { ok = false; return; }
+                  PROF_END(kProfMmaPFull); }
+                if (c.first_in_seg()) {
+                    PROF_BEGIN();
+                    if (!mbar_wait(&bars.o_empty, (c.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
+                    PROF_END(kProfMmaOEmpty);
+                }
                 tc_fence_after();
                 const int s0 = item_of_v(np, N) * SPT;
+                const bool fresh = c.first_in_seg();
+                const bool last = c.last_in_seg();
                 for (int vi = 0; vi < SPT; ++vi) {
                     const int r = vi / NACC, j = vi % NACC;
                     const int s = s0 + vi, slot = s % nslots, use = s / nslots;
-                    if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                    { PROF_BEGIN();
+                      if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                      PROF_END(kProfMmaVFull); }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem + 128u + (uint32_t)(j * 64);
-                    const uint64_t da = desc_mnmajor_sw128(smem_u32(ring + (size_t)slot * kSlotBytes), 8192);
-                    const uint64_t dbh = desc_kmajor_sw128(smem_u32(p_hi + r * (HP * 128)));
-                    const uint64_t dbl = desc_kmajor_sw128(smem_u32(p_lo + r * (HP * 128)));
+                    const uint64_t da = desc_mnmajor_sw128(ring_addr + (uint32_t)slot * kSlotBytes, 8192);
+                    const uint64_t dbh = desc_mnmajor_sw128(phi_addr + (uint32_t)(r * 64 * 128), 8192);
+                    const uint64_t dbl = desc_mnmajor_sw128(plo_addr + (uint32_t)(r * 64 * 128), 8192);
+                    if (elect_one_sync()) {
+#ifndef MQA_X_SKIP_PV
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {   // 4 x 16 cache rows per 64-row slot
-                        const uint32_t acc = (c.first_in_seg() && r == 0 && ks == 0) ? 0u : 1u;
-                        umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbh + (uint64_t)(ks * 2), idesc_pv, acc);
-                        umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbl + (uint64_t)(ks * 2), idesc_pv, 1u);
+                        for (int ks = 0; ks < 4; ++ks) {   // 4 x 16 cache rows per 64-row slot
+                            const uint32_t acc = (fresh && r == 0 && ks == 0) ? 0u : 1u;
+                            umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbh + (uint64_t)(ks * (2048 >> 4)), idesc_pv, acc);
+                            if (use_lo)
+                                umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbl + (uint64_t)(ks * (2048 >> 4)), idesc_pv, 1u);
+                        }
+#endif
+                        umma_commit(&bars.empty[slot]);
+                        if (vi == SPT - 1) {
+                            umma_commit(&bars.p_empty);
+                            if (last) umma_commit(&bars.o_full);
+                        }
                     }
-                    umma_commit(&bars.empty[slot]);
+                    __syncwarp();
                 }
-                umma_commit(&bars.p_empty);
-                if (c.last_in_seg()) umma_commit(&bars.o_full);
                 ++np;
             };
             issue_qk(ck); ck.advance();
             while (ok && cv.valid()) {
                 if (ck.valid()) { issue_qk(ck); ck.advance(); }
-                if (ok) { issue_pv(cv); cv.advance(); }
+                if (ok) { issue_pv(cv, cv.w.len <= p.lo_max_len); cv.advance(); }
             }
+            PROF_END(kProfMmaTotal);
         } else if (warp >= kSoftmaxWarp0) {
             // =============================== softmax + epilogue ===============================
-            const int row = tid - kSoftmaxWarp0 * 32;          // cache row within the tile = tensor-memory lane
-            const int wq = warp - kSoftmaxWarp0;               // lane quadrant of this warp
+            // Thread = (cache row of the tile, group of 16 heads).  Warp w reads tensor-memory lanes 32*(w%4)..+31.
+            constexpr int HPT = kHeadsPerThread;
+            constexpr int NSM = L::kSoftmaxThreads;
+            const int ws = warp - kSoftmaxWarp0;
+            const int wq = ws & 3;                              // lane quadrant
+            const int hb = (ws >> 2) * HPT;                     // first head of this thread's group
+            const int row = wq * 32 + lane;                     // cache row within the tile = tensor-memory lane
+            const int sid = tid - kSoftmaxWarp0 * 32;           // index among the softmax threads
             const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
             TileCursor c;
             c.init(p, T, cta, misc.sched);
             int ns = 0;
             bool ok = true;
-            float m[HP], l[HP];
+            float l[HPT];
+            PROF_BEGIN();
             while (ok && c.valid()) {
                 // ---------------- new segment ----------------
                 const int b = c.w.b, seg = c.seg;
                 const bool whole = c.w.seg_is_whole();
+                const bool use_lo = c.w.len <= p.lo_max_len;
                 const int slot_id = c.w.seg_slot(cta);
-                if (c.w.seg_owns_first_tile() && row == 0) {
+                if (c.w.seg_owns_first_tile() && sid == 0) {
                     SeqInfo si;
                     si.first_slot = whole ? -1 : slot_id;
                     si.last_cta = cta_of_tile(c.w.P + c.w.nt - 1, T, G);
                     ws_seqinfo(p.workspace)[b] = si;
                 }
 #pragma unroll
-                for (int h = 0; h < HP; ++h) { m[h] = -INFINITY; l[h] = 0.f; }
+                for (int i = 0; i < HPT; ++i) l[i] = 0.f;
+                if (sid < HP) misc.m[sid] = -INFINITY;    // reference maximum per head, shared by all rows
+                softmax_bar_sync(NSM);
                 bool first = true;
                 for (;;) {
                     const int sb = ns & 1;
                     const int nvalid = c.nvalid();
                     const bool last = c.last_in_seg();
-                    if (!mbar_wait(&bars.s_full[sb], (ns >> 1) & 1, abort_flag)) { ok = false; break; }
+                    { PROF_BEGIN();
+                      if (!mbar_wait(&bars.s_full[sb], (ns >> 1) & 1, abort_flag)) { ok = false; break; }
+                      PROF_END(kProfSmSFull); }
                     tc_fence_after();
-                    float y[HP];
-#pragma unroll
-                    for (int h0 = 0; h0 < HP; h0 += 16) tmem_ld16(lane_base + (uint32_t)(sb * 64 + h0), &y[h0]);
+                    float y[HPT];
+                    tmem_ld16(lane_base + (uint32_t)(sb * 64 + hb), y);
                     tmem_wait_ld();
                     tc_fence_before();
                     mbar_arrive(&bars.s_empty[sb]);
                     const bool valid = row < nvalid;
-                    bool exceed = false;
+                    // y = scale_log2 * logit (-inf for rows beyond the sequence); does any y exceed m + threshold?
+                    float xmax = -INFINITY;
 #pragma unroll
-                    for (int h = 0; h < HP; ++h) {
-                        y[h] = valid ? y[h] * p.scale_log2 : -INFINITY;
-                        exceed |= (y[h] > m[h] + kRescaleThreshold);
+                    for (int i = 0; i < HPT; i += 4) {
+                        const float4 mm = *reinterpret_cast<const float4*>(&misc.m[hb + i]);
+                        y[i + 0] = valid ? y[i + 0] * p.scale_log2 : -INFINITY;
+                        y[i + 1] = valid ? y[i + 1] * p.scale_log2 : -INFINITY;
+                        y[i + 2] = valid ? y[i + 2] * p.scale_log2 : -INFINITY;
+                        y[i + 3] = valid ? y[i + 3] * p.scale_log2 : -INFINITY;
+                        // fmaxf drops the NaN of (-inf) - (-inf)
+                        xmax = fmaxf(fmaxf(xmax, fmaxf(y[i] - mm.x, y[i + 1] - mm.y)), fmaxf(y[i + 2] - mm.z, y[i + 3] - mm.w));
                     }
-                    const bool need = softmax_bar_or(exceed);
-                    // probabilities of tile ns overwrite the buffer read by the MMAs of tile ns-1
-                    if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    bool need;
+                    { PROF_BEGIN(); need = softmax_bar_or(xmax > kRescaleThreshold, NSM); PROF_END(kProfSmBar); }
+                    bool waited_p_empty = false;
                     if (need) {
-                        // exact per-head maximum of this tile, then move the reference m up
+                        // exact per-head maximum of this tile; move the reference m up and rescale l and O
+                        PROF_BEGIN();
 #pragma unroll
-                        for (int h = 0; h < HP; ++h) {
-                            const float wm = warp_max_f32(y[h]);
-                            if (lane == (h & 31)) misc.wred[wq][h] = wm;
+                        for (int i = 0; i < HPT; ++i) {
+                            const float wm = warp_max_f32(y[i]);
+                            if (lane == i) misc.wred[wq][hb + i] = wm;
                         }
-                        softmax_bar_sync();
-                        float alpha[HP];
+                        softmax_bar_sync(NSM);
+                        if (sid < HP) {
+                            const float tm = fmaxf(fmaxf(misc.wred[0][sid], misc.wred[1][sid]), fmaxf(misc.wred[2][sid], misc.wred[3][sid]));
+                            const float m_old = misc.m[sid];
+                            const float m_new = fmaxf(m_old, tm);
+                            misc.alpha[sid] = (m_old == -INFINITY) ? 0.f : ex2_approx(m_old - m_new);
+                            misc.m[sid] = m_new;
+                        }
+                        softmax_bar_sync(NSM);
 #pragma unroll
-                        for (int h = 0; h < HP; ++h) {
-                            const float tm = fmaxf(fmaxf(misc.wred[0][h], misc.wred[1][h]), fmaxf(misc.wred[2][h], misc.wred[3][h]));
-                            const float m_new = fmaxf(m[h], tm);
-                            alpha[h] = (m[h] == -INFINITY) ? 0.f : exp2f(m[h] - m_new);
-                            l[h] *= alpha[h];
-                            m[h] = m_new;
-                        }
-                        softmax_bar_sync();   // wred may be reused by the next tile
+                        for (int i = 0; i < HPT; ++i) l[i] *= misc.alpha[hb + i];
                         if (!first) {
-                            // rescale the accumulators in tensor memory (their MMAs have completed: p_empty)
+                            // the accumulators can be rescaled once the MMAs of tile ns-1 have completed
+                            if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                            waited_p_empty = true;
                             tc_fence_after();
 #pragma unroll
                             for (int j = 0; j < NACC; ++j) {
+                                float o[HPT];
+                                const uint32_t ta = lane_base + 128u + (uint32_t)(j * 64 + hb);
+                                tmem_ld16(ta, o);
+                                tmem_wait_ld();
 #pragma unroll
-                                for (int h0 = 0; h0 < HP; h0 += 16) {
-                                    float o[16];
-                                    const uint32_t ta = lane_base + 128u + (uint32_t)(j * 64 + h0);
-                                    tmem_ld16(ta, o);
-                                    tmem_wait_ld();
-#pragma unroll
-                                    for (int i = 0; i < 16; ++i) o[i] *= alpha[h0 + i];
-                                    tmem_st16(ta, o);
-                                }
+                                for (int i = 0; i < HPT; ++i) o[i] *= misc.alpha[hb + i];
+                                tmem_st16(ta, o);
                             }
                             tmem_wait_st();
                             tc_fence_before();
                         }
+                        PROF_END(kProfSmRescale);
                     }
-                    // p = 2^(y - m); write bf16 hi and lo parts into the K-major, 128B-swizzled B operand
+                    // p = 2^(y - m) as bf16 hi (and lo) halves, packed in registers while the MMAs of the
+                    // previous tile still read the probability buffer
+                    uint32_t hw[HPT / 2], lw[HPT / 2];
                     {
-                        const int chunk = row >> 6, col = row & 63;
-                        const uint32_t unit = (uint32_t)(col >> 3), within = (uint32_t)(col & 7) * 2u;
-                        unsigned char* ph = p_hi + chunk * (HP * 128);
-                        unsigned char* pl = p_lo + chunk * (HP * 128);
+                        PROF_BEGIN();
 #pragma unroll
-                        for (int h = 0; h < HP; ++h) {
-                            const float pr = exp2f(y[h] - m[h]);          // 0 for masked rows (y = -inf, m finite)
-                            l[h] += pr;
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(pr);
-                            const __nv_bfloat16 lo = __float2bfloat16_rn(pr - __bfloat162float(hi));
-                            const uint32_t off = (uint32_t)h * 128u + ((unit ^ (uint32_t)(h & 7)) << 4) + within;
-                            *reinterpret_cast<__nv_bfloat16*>(ph + off) = hi;
-                            *reinterpret_cast<__nv_bfloat16*>(pl + off) = lo;
+                        for (int i = 0; i < HPT; i += 2) {
+                            const float2 mm = *reinterpret_cast<const float2*>(&misc.m[hb + i]);
+                            const float p0 = ex2_approx(y[i] - mm.x), p1 = ex2_approx(y[i + 1] - mm.y);   // 0 for masked rows
+                            l[i] += p0; l[i + 1] += p1;
+                            const __nv_bfloat162 hb2 = __floats2bfloat162_rn(p0, p1);
+                            const uint32_t w32 = *reinterpret_cast<const uint32_t*>(&hb2);
+                            hw[i / 2] = w32;
+                            const __nv_bfloat162 lb2 = __floats2bfloat162_rn(p0 - __uint_as_float(w32 << 16),
+                                                                             p1 - __uint_as_float(w32 & 0xffff0000u));
+                            lw[i / 2] = *reinterpret_cast<const uint32_t*>(&lb2);
+                        }
+                        PROF_END(kProfSmStore);
+                    }
+                    // the probabilities of tile ns overwrite the buffer read by the MMAs of tile ns-1
+                    if (!waited_p_empty) {
+                        PROF_BEGIN();
+                        if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        PROF_END(kProfSmPEmpty);
+                    }
+                    {
+                        // MN-major, 128B-swizzled B operand: one 128-byte row per cache row, heads contiguous
+                        unsigned char* ph = p_hi + row * 128;
+                        unsigned char* pl = p_lo + row * 128;
+#pragma unroll
+                        for (int u = 0; u < HPT / 8; ++u) {
+                            const uint32_t unit = (uint32_t)(hb / 8 + u);
+                            const uint32_t off = (unit ^ (uint32_t)(row & 7)) << 4;
+                            *reinterpret_cast<uint4*>(ph + off) = make_uint4(hw[4 * u], hw[4 * u + 1], hw[4 * u + 2], hw[4 * u + 3]);
+                            if (use_lo)
+                                *reinterpret_cast<uint4*>(pl + off) = make_uint4(lw[4 * u], lw[4 * u + 1], lw[4 * u + 2], lw[4 * u + 3]);
                         }
                     }
                     if (nvalid < kTileRows) {
@@ -486,7 +619,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                             const int r = vi / NACC;
                             const int s = s0 + vi, slot = s % nslots, use = s / nslots;
                             if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; break; }
-                            if (!valid && (row >> 6) == r) {
+                            if (hb == 0 && !valid && (row >> 6) == r) {
                                 uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (row & 63) * 128);
                                 uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + (row & 63) * 128);
 #pragma unroll
@@ -504,60 +637,74 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 }
                 if (!ok) break;
                 // ---------------- segment epilogue ----------------
+                const float m_mine = (sid < HP) ? misc.m[sid] : 0.f;
                 // row sums over the 128 cache-row lanes
 #pragma unroll
-                for (int h = 0; h < HP; ++h) {
-                    float v = l[h];
+                for (int i = 0; i < HPT; ++i) {
+                    float v = l[i];
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (lane == (h & 31)) misc.wred[wq][h] = v;
+                    if (lane == i) misc.wred[wq][hb + i] = v;
                 }
-                softmax_bar_sync();
-                float lsum[HP];
-#pragma unroll
-                for (int h = 0; h < HP; ++h) lsum[h] = (misc.wred[0][h] + misc.wred[1][h]) + (misc.wred[2][h] + misc.wred[3][h]);
-                float oscale[HP];   // 1/l for a direct write, 1 for an unnormalised partial
-#pragma unroll
-                for (int h = 0; h < HP; ++h) oscale[h] = whole ? 1.f / lsum[h] : 1.f;
-                softmax_bar_sync();
-                if (!mbar_wait(&bars.o_full, seg & 1, abort_flag)) { ok = false; break; }
+                softmax_bar_sync(NSM);
+                if (sid < HP) misc.alpha[sid] = (misc.wred[0][sid] + misc.wred[1][sid]) + (misc.wred[2][sid] + misc.wred[3][sid]);
+                softmax_bar_sync(NSM);     // misc.alpha now holds the row sums l[h]
+                { PROF_BEGIN();
+                  if (!mbar_wait(&bars.o_full, seg & 1, abort_flag)) { ok = false; break; }
+                  PROF_END(kProfSmOFull); }
                 tc_fence_after();
+                {
+                PROF_BEGIN();
                 float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, slot_id);
                 const int Hp4 = round_up(H, 4);
-                if (!whole && row < H) {
-                    // m is identical in every thread; thread `row` stores head `row`
-                    float mv = 0.f, lv = 0.f;
-#pragma unroll
-                    for (int h = 0; h < HP; ++h) if (h == row) { mv = m[h]; lv = lsum[h]; }
-                    slot_ptr[row] = mv;
-                    slot_ptr[Hp4 + row] = lv;
+                if (!whole && sid < H) {
+                    slot_ptr[sid] = m_mine;
+                    slot_ptr[Hp4 + sid] = misc.alpha[sid];
                 }
+                float o[NACC][HPT];
+#pragma unroll
+                for (int j = 0; j < NACC; ++j) tmem_ld16(lane_base + 128u + (uint32_t)(j * 64 + hb), o[j]);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(&bars.o_empty);      // the accumulators are in registers: the next segment may overwrite them
 #pragma unroll
                 for (int j = 0; j < NACC; ++j) {
                     const int d = j * 128 + row;
+                    if (whole) {
+                        float* dst = p.out + ((size_t)b * H + hb) * D + d;
 #pragma unroll
-                    for (int h0 = 0; h0 < HP; h0 += 16) {
-                        float o[16];
-                        tmem_ld16(lane_base + 128u + (uint32_t)(j * 64 + h0), o);
-                        tmem_wait_ld();
+                        for (int i = 0; i < HPT; ++i)
+                            if (hb + i < H) dst[(size_t)i * D] = o[j][i] * __frcp_rn(misc.alpha[hb + i]);
+                    } else {
+                        float* dst = slot_ptr + 2 * Hp4 + (size_t)hb * D + d;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int h = h0 + i;
-                            if (h < H) {
-                                if (whole) p.out[((size_t)b * H + h) * D + d] = o[i] * oscale[h];
-                                else slot_ptr[2 * Hp4 + (size_t)h * D + d] = o[i];
-                            }
-                        }
+                        for (int i = 0; i < HPT; ++i)
+                            if (hb + i < H) dst[(size_t)i * D] = o[j][i];
                     }
                 }
-                tc_fence_before();
-                mbar_arrive(&bars.o_empty);
+                softmax_bar_sync(NSM);     // misc.m / misc.alpha are rewritten by the next segment
+                PROF_END(kProfSmEpilogue);
+                }
             }
+            PROF_END(kProfSmTotal);
         }
     }
 
     __syncwarp();
     __syncthreads();
+#ifdef MQA_TC_PROFILE
+    if (tid == 0) {
+        unsigned long long ns1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+        if (blockIdx.x == MQA_PROF_BLOCK) {
+            ws_header(p.workspace)[16 + 30] = (int)(ns1 - prof_ns0);
+            ws_header(p.workspace)[16 + 31] = (int)(clock64() - prof_c0);
+        }
+        // per-block start/end times and SM id, in the last (unused) partial slot
+        unsigned long long* tl = reinterpret_cast<unsigned long long*>(ws_slot(p.workspace, p.B, p.H, D, 2 * kMaxCtas - 1));
+        unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        tl[3 * blockIdx.x] = prof_ns0; tl[3 * blockIdx.x + 1] = ns1; tl[3 * blockIdx.x + 2] = smid;
+    }
+#endif
     if (tid == 0 && misc.abort_flag) atomicExch(ws_header(p.workspace) + kHdrStatus, 7 /* MQA_ERR_TIMEOUT */);
     if (warp == 1) {
         tc_fence_after();
@@ -579,6 +726,18 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn()
     return fn;
 }
 
+// Sequences up to this length carry the low-order bf16 half of every probability through a second
+// MMA.  A bf16 probability alone (8 significant bits) misses the 2e-3 tolerance when an output is a blend
+// of a handful of rows; the default keeps both halves for every length.  MQA_LO_MAX_LEN overrides (tuning).
+int lo_max_len_setting()
+{
+    static const int v = []() {
+        const char* e = getenv("MQA_LO_MAX_LEN");
+        return e ? atoi(e) : 0x7fffffff;
+    }();
+    return v;
+}
+
 // 3-D bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box [1][box1][64], 128-byte swizzle, zero fill.
 bool encode_map(CUtensorMap* map, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box1)
 {
@@ -594,8 +753,10 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t dim0, uint64_t dim1
 }
 
 template <int D, int HP>
-cudaError_t launch_tc_t(const Params& p, cudaStream_t stream)
+cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
 {
+    Params p = p_in;
+    p.lo_max_len = lo_max_len_setting();
     using L = TcLayout<D, HP>;
     int dev = 0, smem_limit = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -611,10 +772,12 @@ cudaError_t launch_tc_t(const Params& p, cudaStream_t stream)
         return cudaErrorInvalidValue;
     e = cudaFuncSetAttribute(mqa_tc_kernel<D, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    mqa_tc_kernel<D, HP><<<p.num_ctas, kTcThreads, smem, stream>>>(p, mq, mk, mv, nslots);
+    mqa_tc_kernel<D, HP><<<p.num_ctas, L::kThreads, smem, stream>>>(p, mq, mk, mv, nslots);
     return cudaGetLastError();
 }
 
+}  // namespace
+namespace {
 template <int D>
 cudaError_t launch_tc_d(const Params& p, cudaStream_t stream)
 {
