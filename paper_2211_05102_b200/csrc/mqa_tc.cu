@@ -70,6 +70,15 @@ struct Misc {
 #define PROF_BEGIN() do {} while (0)
 #define PROF_END(idx) do {} while (0)
 #endif
+// Optional event trace (compile with -DMQA_TC_TRACE=<block>): one elected thread per role appends
+// (event id, tile counter, clock) records for that block to the last, unused partial slot.
+#ifdef MQA_TC_TRACE
+#define TRACE(role, id, n) do { if (blockIdx.x == MQA_TC_TRACE && (threadIdx.x & 31) == 0) { \
+    long long* tb_ = reinterpret_cast<long long*>(ws_slot(p.workspace, p.B, p.H, D, 2 * kMaxCtas - 2)) + (role) * 2048; \
+    if (trace_n < 1000) { tb_[2 * trace_n] = ((long long)(id) << 32) | (unsigned)(n); tb_[2 * trace_n + 1] = clock64(); ++trace_n; } } } while (0)
+#else
+#define TRACE(role, id, n) do {} while (0)
+#endif
 enum { kProfProdEmpty = 0, kProfMmaSEmpty, kProfMmaQFull, kProfMmaKFull, kProfMmaPFull, kProfMmaOEmpty, kProfMmaVFull,
        kProfSmSFull, kProfSmBar, kProfSmPEmpty, kProfSmRescale, kProfSmStore, kProfSmEpilogue, kProfSmTotal, kProfMmaTotal,
        kProfProdTotal, kProfSmLoad, kProfSmOFull };
@@ -86,6 +95,8 @@ __device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(void* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One probe of the barrier (measured on B200: the form with a suspend-time hint costs ~45 cycles more per
+// hand-off than this one, so it is not used).
 __device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -312,9 +323,13 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             ck.init(p, T, cta, misc.sched);
             cv = ck;
             int slot_seq = 0;          // running slot counter = item * SPT + chunk
+            int pslot = 0;             // slot_seq % nslots
+            uint32_t pphase = 0;       // (slot_seq / nslots) & 1
             bool ok = true;
+            int trace_n = 0; (void)trace_n;
             PROF_BEGIN();
             auto load_k = [&](const TileCursor& c) {
+#ifndef MQA_X_LOADONLY
                 if (c.first_in_seg()) {   // stage this sequence's queries first
                     const int qb = c.seg & 1;
                     if (!mbar_wait(&bars.q_empty[qb], ((c.seg >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
@@ -325,38 +340,53 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     }
                     __syncwarp();
                 }
+#endif
+#pragma unroll
                 for (int ch = 0; ch < SPT; ++ch) {
-                    const int slot = slot_seq % nslots, use = slot_seq / nslots;
+                    const int slot = pslot;
                     {
                         PROF_BEGIN();
-                        if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return; }
+                        if (!mbar_wait(&bars.empty[slot], pphase ^ 1, abort_flag)) { ok = false; return; }
                         PROF_END(kProfProdEmpty);
                     }
+                    TRACE(0, 1, slot_seq);
                     if (elect_one_sync()) {
+#ifdef MQA_X_NOLOAD
+                        mbar_arrive(&bars.full[slot]);
+#else
                         mbar_expect_tx(&bars.full[slot], kSlotBytes);
                         tma_load_3d(ring + (size_t)slot * kSlotBytes, &map_k, &bars.full[slot], ch * 64, c.row0(), c.w.b, policy);
+#endif
                     }
                     __syncwarp();
                     ++slot_seq;
+                    if (++pslot == nslots) { pslot = 0; pphase ^= 1; }
                 }
             };
             auto load_v = [&](const TileCursor& c) {
+#pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
                     const int r = vi / NACC, j = vi % NACC;
-                    const int slot = slot_seq % nslots, use = slot_seq / nslots;
+                    const int slot = pslot;
                     {
                         PROF_BEGIN();
-                        if (!mbar_wait(&bars.empty[slot], (use & 1) ^ 1, abort_flag)) { ok = false; return; }
+                        if (!mbar_wait(&bars.empty[slot], pphase ^ 1, abort_flag)) { ok = false; return; }
                         PROF_END(kProfProdEmpty);
                     }
+                    TRACE(0, 2, slot_seq);
                     if (elect_one_sync()) {
                         unsigned char* dst = ring + (size_t)slot * kSlotBytes;
+#ifdef MQA_X_NOLOAD
+                        (void)dst; mbar_arrive(&bars.full[slot]);
+#else
                         mbar_expect_tx(&bars.full[slot], kSlotBytes);
                         tma_load_3d(dst, &map_v, &bars.full[slot], j * 128, c.row0() + r * 64, c.w.b, policy);
                         tma_load_3d(dst + 8192, &map_v, &bars.full[slot], j * 128 + 64, c.row0() + r * 64, c.w.b, policy);
+#endif
                     }
                     __syncwarp();
                     ++slot_seq;
+                    if (++pslot == nslots) { pslot = 0; pphase ^= 1; }
                 }
             };
             load_k(ck); ck.advance();
@@ -381,9 +411,15 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             ck.init(p, T, cta, misc.sched);
             cv = ck;
             int nq = 0, np = 0;
+            int cslot = 0;             // ring slot consumed next: slots are used in the order they were filled
+            uint32_t cphase = 0;
             bool ok = true;
-            const uint32_t ring_addr = smem_u32(ring), q_addr = smem_u32(q_buf);
-            const uint32_t phi_addr = smem_u32(p_hi), plo_addr = smem_u32(p_lo);
+            int trace_n = 0; (void)trace_n;
+            const uint32_t q_addr = smem_u32(q_buf);
+            const uint64_t desc_ring0 = desc_kmajor_sw128(smem_u32(ring));
+            const uint64_t desc_ring0_mn = desc_mnmajor_sw128(smem_u32(ring), 8192);
+            const uint64_t desc_phi = desc_mnmajor_sw128(smem_u32(p_hi), 8192);
+            const uint64_t desc_plo = desc_mnmajor_sw128(smem_u32(p_lo), 8192);
             PROF_BEGIN();
             auto issue_qk = [&](const TileCursor& c) {
                 const int sb = nq & 1;
@@ -397,15 +433,20 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     PROF_END(kProfMmaQFull);
                 }
                 const uint32_t d_tmem = tmem + (uint32_t)(sb * 64);
-                const int s0 = item_of_k(nq) * SPT;
+                const uint64_t db0 = desc_kmajor_sw128(q_addr + (uint32_t)(qb * L::kQBytes));
+                const bool last = c.last_in_seg();
+                TRACE(1, 10, nq);   // QK: s_empty and q ready
+#pragma unroll
                 for (int ch = 0; ch < SPT; ++ch) {
-                    const int s = s0 + ch, slot = s % nslots, use = s / nslots;
+                    const int slot = cslot;
                     { PROF_BEGIN();
-                      if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                      if (!mbar_wait(&bars.full[slot], cphase, abort_flag)) { ok = false; return; }
                       PROF_END(kProfMmaKFull); }
+                    if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
                     tc_fence_after();
-                    const uint64_t da = desc_kmajor_sw128(ring_addr + (uint32_t)slot * kSlotBytes);
-                    const uint64_t db = desc_kmajor_sw128(q_addr + (uint32_t)(qb * L::kQBytes + ch * (HP * 128)));
+                    TRACE(1, 11 + ch, nq);   // K chunk landed
+                    const uint64_t da = desc_ring0 + (uint64_t)((uint32_t)slot * (kSlotBytes >> 4));
+                    const uint64_t db = db0 + (uint64_t)(ch * (HP * 128 >> 4));
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_QK
 #pragma unroll
@@ -415,11 +456,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         umma_commit(&bars.empty[slot]);
                         if (ch == SPT - 1) {
                             umma_commit(&bars.s_full[sb]);
-                            if (c.last_in_seg()) umma_commit(&bars.q_empty[qb]);
+                            if (last) umma_commit(&bars.q_empty[qb]);
                         }
                     }
                     __syncwarp();
                 }
+                TRACE(1, 15, nq);   // QK issued
                 ++nq;
             };
             auto issue_pv = [&](const TileCursor& c, bool use_lo) {
@@ -432,20 +474,23 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     PROF_END(kProfMmaOEmpty);
                 }
                 tc_fence_after();
-                const int s0 = item_of_v(np, N) * SPT;
+                TRACE(1, 20, np);   // P ready
                 const bool fresh = c.first_in_seg();
                 const bool last = c.last_in_seg();
+#pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
                     const int r = vi / NACC, j = vi % NACC;
-                    const int s = s0 + vi, slot = s % nslots, use = s / nslots;
+                    const int slot = cslot;
                     { PROF_BEGIN();
-                      if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; return; }
+                      if (!mbar_wait(&bars.full[slot], cphase, abort_flag)) { ok = false; return; }
                       PROF_END(kProfMmaVFull); }
+                    if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
                     tc_fence_after();
+                    TRACE(1, 21 + vi, np);   // V slot landed
                     const uint32_t d_tmem = tmem + 128u + (uint32_t)(j * 64);
-                    const uint64_t da = desc_mnmajor_sw128(ring_addr + (uint32_t)slot * kSlotBytes, 8192);
-                    const uint64_t dbh = desc_mnmajor_sw128(phi_addr + (uint32_t)(r * 64 * 128), 8192);
-                    const uint64_t dbl = desc_mnmajor_sw128(plo_addr + (uint32_t)(r * 64 * 128), 8192);
+                    const uint64_t da = desc_ring0_mn + (uint64_t)((uint32_t)slot * (kSlotBytes >> 4));
+                    const uint64_t dbh = desc_phi + (uint64_t)(r * (64 * 128 >> 4));
+                    const uint64_t dbl = desc_plo + (uint64_t)(r * (64 * 128 >> 4));
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_PV
 #pragma unroll
@@ -464,13 +509,24 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     }
                     __syncwarp();
                 }
+                TRACE(1, 25, np);   // PV issued
                 ++np;
             };
+#ifdef MQA_X_LOADONLY
+            // experiment: free every slot as soon as it has landed (measures the staging rate alone)
+            for (int s = 0; s < 2 * N * SPT && ok; ++s) {
+                const int slot = s % nslots, use = s / nslots;
+                if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; break; }
+                if (elect_one_sync()) mbar_arrive(&bars.empty[slot]);
+                __syncwarp();
+            }
+#else
             issue_qk(ck); ck.advance();
             while (ok && cv.valid()) {
                 if (ck.valid()) { issue_qk(ck); ck.advance(); }
                 if (ok) { issue_pv(cv, cv.w.len <= p.lo_max_len); cv.advance(); }
             }
+#endif
             PROF_END(kProfMmaTotal);
         } else if (warp >= kSoftmaxWarp0) {
             // =============================== softmax + epilogue ===============================
@@ -488,7 +544,22 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             int ns = 0;
             bool ok = true;
             float l[HPT];
+            int trace_n = (ws == 0) ? 0 : 100000; (void)trace_n;
+            // Only the first softmax warp watches an mbarrier; the others are released through the named
+            // barrier, which also makes the outcome uniform across the group.
+            auto group_wait = [&](void* bar, uint32_t parity) -> bool {
+#ifdef MQA_GROUP_WAIT_ALL
+                return mbar_wait(bar, parity, abort_flag);
+#else
+                bool failed = false;
+                if (ws == 0) failed = !mbar_wait(bar, parity, abort_flag);
+                return !softmax_bar_or(failed, NSM);
+#endif
+            };
             PROF_BEGIN();
+#ifdef MQA_X_LOADONLY
+            ok = false;
+#endif
             while (ok && c.valid()) {
                 // ---------------- new segment ----------------
                 const int b = c.w.b, seg = c.seg;
@@ -511,9 +582,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     const int nvalid = c.nvalid();
                     const bool last = c.last_in_seg();
                     { PROF_BEGIN();
-                      if (!mbar_wait(&bars.s_full[sb], (ns >> 1) & 1, abort_flag)) { ok = false; break; }
+                      if (!group_wait(&bars.s_full[sb], (ns >> 1) & 1)) { ok = false; break; }
                       PROF_END(kProfSmSFull); }
                     tc_fence_after();
+                    TRACE(2, 30, ns);   // S ready
                     float y[HPT];
                     tmem_ld16(lane_base + (uint32_t)(sb * 64 + hb), y);
                     tmem_wait_ld();
@@ -534,6 +606,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     }
                     bool need;
                     { PROF_BEGIN(); need = softmax_bar_or(xmax > kRescaleThreshold, NSM); PROF_END(kProfSmBar); }
+                    TRACE(2, 31, ns);   // after bar.red
                     bool waited_p_empty = false;
                     if (need) {
                         // exact per-head maximum of this tile; move the reference m up and rescale l and O
@@ -556,7 +629,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         for (int i = 0; i < HPT; ++i) l[i] *= misc.alpha[hb + i];
                         if (!first) {
                             // the accumulators can be rescaled once the MMAs of tile ns-1 have completed
-                            if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                            if (!group_wait(&bars.p_empty, (ns & 1) ^ 1)) { ok = false; break; }
                             waited_p_empty = true;
                             tc_fence_after();
 #pragma unroll
@@ -593,12 +666,14 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         }
                         PROF_END(kProfSmStore);
                     }
+                    TRACE(2, 32, ns);   // p packed
                     // the probabilities of tile ns overwrite the buffer read by the MMAs of tile ns-1
                     if (!waited_p_empty) {
                         PROF_BEGIN();
-                        if (!mbar_wait(&bars.p_empty, (ns & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        if (!group_wait(&bars.p_empty, (ns & 1) ^ 1)) { ok = false; break; }
                         PROF_END(kProfSmPEmpty);
                     }
+                    TRACE(2, 33, ns);   // p_empty seen
                     {
                         // MN-major, 128B-swizzled B operand: one 128-byte row per cache row, heads contiguous
                         unsigned char* ph = p_hi + row * 128;
@@ -618,7 +693,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         for (int vi = 0; vi < SPT; ++vi) {
                             const int r = vi / NACC;
                             const int s = s0 + vi, slot = s % nslots, use = s / nslots;
-                            if (!mbar_wait(&bars.full[slot], use & 1, abort_flag)) { ok = false; break; }
+                            if (!group_wait(&bars.full[slot], use & 1)) { ok = false; break; }
                             if (hb == 0 && !valid && (row >> 6) == r) {
                                 uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (row & 63) * 128);
                                 uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + (row & 63) * 128);
@@ -630,6 +705,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     }
                     fence_proxy_async();
                     mbar_arrive(&bars.p_full);
+                    TRACE(2, 34, ns);   // P published
                     first = false;
                     ++ns;
                     c.advance();
@@ -650,7 +726,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 if (sid < HP) misc.alpha[sid] = (misc.wred[0][sid] + misc.wred[1][sid]) + (misc.wred[2][sid] + misc.wred[3][sid]);
                 softmax_bar_sync(NSM);     // misc.alpha now holds the row sums l[h]
                 { PROF_BEGIN();
-                  if (!mbar_wait(&bars.o_full, seg & 1, abort_flag)) { ok = false; break; }
+                  if (!group_wait(&bars.o_full, seg & 1)) { ok = false; break; }
                   PROF_END(kProfSmOFull); }
                 tc_fence_after();
                 {
