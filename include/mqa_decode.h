@@ -83,7 +83,8 @@ const char* mqa_status_string(int status);
 /*
  * Bytes of device workspace mqa_decode needs for this shape under ANY plan the
  * library may choose: a 256-byte header (device status word, tile total), one
- * 8-byte record per sequence, and two partial-result slots per thread block
+ * 8-byte record and one 4-byte arrival counter per sequence (each array rounded
+ * up to 256 bytes), and two partial-result slots per thread block
  * (per slot: running max and running sum per head, and the unnormalised fp32
  * accumulator [H,D]).  Returns 0 for an unsupported shape.  Host-only; no
  * device is touched.
@@ -91,8 +92,10 @@ const char* mqa_status_string(int status);
 size_t mqa_decode_workspace_bytes(int B, int H, int D, int Lmax);
 
 /*
- * Zero the workspace header (the device status word).  Call once after
- * allocating the workspace, before the first mqa_decode that uses it.
+ * Zero the workspace (device status word, per-sequence records and arrival
+ * counters must start at zero; the kernels leave them zero again).  Call once
+ * after allocating the workspace, before the first mqa_decode that uses it,
+ * and again after a call that reported MQA_ERR_TIMEOUT.
  */
 int mqa_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
@@ -182,7 +185,7 @@ int mqa_last_launch_count(void);
  *
  * Arguments, layouts and results are those of mqa_decode, without the
  * workspace.  Limits: the shape must fit the fixed array, i.e.
- *   256 + roundup(8*B, 256) + 2 * 4*(2*roundup(H,4) + H*D) <= MQA_STATIC_WORKSPACE_BYTES;
+ *   256 + roundup(8*B, 256) + roundup(4*B, 256) + 2 * 4*(2*roundup(H,4) + H*D) <= MQA_STATIC_WORKSPACE_BYTES;
  * a larger shape returns MQA_ERR_WORKSPACE_TOO_SMALL and launches nothing.
  * When the heuristic's block count would not fit, fewer blocks are used.
  * The call makes no cudaMalloc/cudaFree and uses no allocating library
@@ -191,8 +194,8 @@ int mqa_last_launch_count(void);
  * any stream capture.
  *
  * All calls on one device share the array, and it keeps the last call's
- * contents: the call clears the part that must start at zero (the header) on
- * `stream` before launching.  Calls whose kernels may overlap on the GPU
+ * contents: the call clears the part that must start at zero (header, records,
+ * counters) on `stream` before launching.  Calls whose kernels may overlap on the GPU
  * (different streams without ordering) race on the array; order them.  A
  * time-out of a bounded device-side wait cannot be read back through this
  * entry point; use mqa_decode with mqa_check_status to diagnose one.

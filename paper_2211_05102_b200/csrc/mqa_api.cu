@@ -62,7 +62,8 @@ int mqa_workspace_init(void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!workspace) return MQA_ERR_INVALID_ARG;
     if (workspace_bytes < (size_t)mqa::kHeaderBytes) return MQA_ERR_WORKSPACE_TOO_SMALL;
-    if (cudaMemsetAsync(workspace, 0, mqa::kHeaderBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    const size_t n = workspace_bytes;   // header, per-sequence records and arrival counters must start at zero
+    if (cudaMemsetAsync(workspace, 0, n, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MQA_ERR_CUDA;
     return MQA_OK;
 }
@@ -137,9 +138,12 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     if (e != cudaSuccess) return MQA_ERR_CUDA;
     if (event_after_split && cudaEventRecord(static_cast<cudaEvent_t>(event_after_split), st) != cudaSuccess)
         return MQA_ERR_CUDA;
-    e = mqa::launch_combine(p, st);
-    if (e != cudaSuccess) return MQA_ERR_CUDA;
-    g_last_launches = 2;
+    g_last_launches = 1;
+    if (plan->path != MQA_PATH_TC) {   // the tensor-core kernel merges cut sequences itself
+        e = mqa::launch_combine(p, st);
+        if (e != cudaSuccess) return MQA_ERR_CUDA;
+        g_last_launches = 2;
+    }
     return MQA_OK;
 }
 

@@ -38,8 +38,13 @@ __host__ __device__ inline size_t slot_floats(int H, int D) {
     return (size_t)2 * round_up(H, 4) + (size_t)H * D;
 }
 __host__ __device__ inline size_t seqinfo_offset() { return kHeaderBytes; }
-__host__ __device__ inline size_t slots_offset(int B) {
+// One arrival counter per sequence (tensor-core path: the block that delivers the last partial result of a
+// cut sequence merges them).  Zero between calls: the merging block resets it.
+__host__ __device__ inline size_t arrivals_offset(int B) {
     return kHeaderBytes + ((size_t)B * sizeof(SeqInfo) + 255) / 256 * 256;
+}
+__host__ __device__ inline size_t slots_offset(int B) {
+    return arrivals_offset(B) + ((size_t)B * sizeof(int) + 255) / 256 * 256;
 }
 __host__ __device__ inline size_t workspace_bytes(int B, int H, int D) {
     return slots_offset(B) + (size_t)2 * kMaxCtas * slot_floats(H, D) * sizeof(float);
@@ -64,6 +69,9 @@ __host__ __device__ __forceinline__ int clamp_len(int len, int Lmax) { return le
 __device__ __forceinline__ int* ws_header(unsigned char* ws) { return reinterpret_cast<int*>(ws); }
 __device__ __forceinline__ SeqInfo* ws_seqinfo(unsigned char* ws) {
     return reinterpret_cast<SeqInfo*>(ws + seqinfo_offset());
+}
+__device__ __forceinline__ int* ws_arrivals(unsigned char* ws, int B) {
+    return reinterpret_cast<int*>(ws + arrivals_offset(B));
 }
 __device__ __forceinline__ float* ws_slot(unsigned char* ws, int B, int H, int D, int slot) {
     return reinterpret_cast<float*>(ws + slots_offset(B)) + (size_t)slot * slot_floats(H, D);

@@ -10,8 +10,9 @@
 // and shapes that would need more are rejected.
 //
 // All calls on a device share the one array, and the array keeps whatever the last
-// call left in it.  The only part that must start clean is the header (the device
-// status word), which each call clears on its stream before launching.  Two calls
+// call left in it.  The parts that must start clean (the header with the device status
+// word, the per-sequence records and arrival counters) are cleared by each call on its
+// stream before launching.  Two calls
 // whose kernels overlap on the GPU (different streams, no ordering) would race on
 // the array: callers must order them.
 #include "../../include/mqa_decode.h"
@@ -87,8 +88,9 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     if (rc != MQA_OK) return rc;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // The array keeps the previous call's contents; only the header has to start at zero.
-    if (cudaMemsetAsync(ws, 0, mqa::kHeaderBytes, st) != cudaSuccess) return MQA_ERR_CUDA;
+    // The array keeps the previous call's contents; the header, the per-sequence records and the arrival
+    // counters (everything in front of the partial-result slots) have to start at zero.
+    if (cudaMemsetAsync(ws, 0, fixed, st) != cudaSuccess) return MQA_ERR_CUDA;
 
     mqa::Params p;
     p.q = static_cast<const uint16_t*>(q);
@@ -104,6 +106,6 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     p.workspace = ws;
     cudaError_t e = (plan.path == MQA_PATH_TC) ? mqa::launch_tc(p, st) : mqa::launch_fma(p, st);
     if (e != cudaSuccess) return MQA_ERR_CUDA;
-    if (mqa::launch_combine(p, st) != cudaSuccess) return MQA_ERR_CUDA;
+    if (plan.path != MQA_PATH_TC && mqa::launch_combine(p, st) != cudaSuccess) return MQA_ERR_CUDA;
     return MQA_OK;
 }

@@ -52,6 +52,9 @@ struct Misc {
     SchedShared sched;
     uint32_t tmem_base;
     int abort_flag;
+    int n_pending;                 // cut sequences whose last partial result this block delivered
+    int pending[2];                // (a block has at most two partial segments)
+    int pending_p[2], pending_nt[2];   // first global tile and tile count of those sequences
     float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
     __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
     __align__(16) float alpha[kMaxHeads];  // rescale factors; row sums in the epilogue
@@ -245,6 +248,88 @@ struct TileCursor {
 __device__ __forceinline__ int item_of_k(int n) { return n == 0 ? 0 : 2 * n - 1; }
 __device__ __forceinline__ int item_of_v(int n, int N) { return n == N - 1 ? 2 * N - 1 : 2 * n + 2; }
 
+// Log-sum-exp merge of the partial results of one cut sequence, by every thread of the block:
+//   M = max_s m_s;  out = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s
+// Parts are folded in block order with a running maximum, so the result does not depend on which
+// block performs the merge.  A thread owns GR float4 groups of the [H, D] output at a time and keeps the
+// loads of PU parts in flight together (the merge is bound by round trips to L2, not by bytes).
+template <int D, int GR, int PU>
+__device__ __forceinline__ void merge_parts(const Params& p, int T, int b, int i_first, int first_slot, int last_cta, int nthreads)
+{
+    const int H = p.H, G = p.num_ctas, Hp4 = round_up(H, 4);
+    const int total = H * D / 4;                       // float4 groups of the output
+    for (int base = 0; base < total; base += nthreads * GR) {
+        float M[GR], Ls[GR];
+        float4 acc[GR];
+#pragma unroll
+        for (int g = 0; g < GR; ++g) { M[g] = -INFINITY; Ls[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
+        int i2 = i_first;
+        while (i2 <= last_cta) {
+            const float* sp[PU];
+            int np = 0;
+#pragma unroll
+            for (int u = 0; u < PU; ++u) sp[u] = nullptr;
+#pragma unroll
+            for (int u = 0; u < PU; ++u) {
+                // next block in [i2, last_cta] that owns tiles
+                while (i2 <= last_cta && i2 > i_first && span_begin(i2, T, G) == span_begin(i2 + 1, T, G)) ++i2;
+                if (i2 <= last_cta) { sp[u] = ws_slot(p.workspace, p.B, H, D, i2 == i_first ? first_slot : 2 * i2); ++i2; ++np; }
+            }
+            float ms[PU][GR], ls[PU][GR];
+            float4 as[PU][GR];
+#pragma unroll
+            for (int u = 0; u < PU; ++u) {
+#pragma unroll
+                for (int g = 0; g < GR; ++g) {
+                    const int e = base + g * nthreads + (int)threadIdx.x;
+                    if (u < np && e < total) {
+                        const int h = (e * 4) / D;
+                        ms[u][g] = __ldcg(sp[u] + h);
+                        ls[u][g] = __ldcg(sp[u] + Hp4 + h);
+                        as[u][g] = __ldcg(reinterpret_cast<const float4*>(sp[u] + 2 * Hp4) + e);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < PU; ++u) {
+#pragma unroll
+                for (int g = 0; g < GR; ++g) {
+                    const int e = base + g * nthreads + (int)threadIdx.x;
+                    if (u < np && e < total) {
+                        const float m_new = fmaxf(M[g], ms[u][g]);
+                        const float wa = (M[g] == -INFINITY) ? 0.f : ex2_approx(M[g] - m_new);
+                        const float wb = ex2_approx(ms[u][g] - m_new);
+                        M[g] = m_new;
+                        Ls[g] = fmaf(wa, Ls[g], wb * ls[u][g]);
+                        acc[g].x = fmaf(wa, acc[g].x, wb * as[u][g].x); acc[g].y = fmaf(wa, acc[g].y, wb * as[u][g].y);
+                        acc[g].z = fmaf(wa, acc[g].z, wb * as[u][g].z); acc[g].w = fmaf(wa, acc[g].w, wb * as[u][g].w);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < GR; ++g) {
+            const int e = base + g * nthreads + (int)threadIdx.x;
+            if (e < total) {
+                const float inv = __frcp_rn(Ls[g]);
+                reinterpret_cast<float4*>(p.out + (size_t)b * H * D)[e] =
+                    make_float4(acc[g].x * inv, acc[g].y * inv, acc[g].z * inv, acc[g].w * inv);
+            }
+        }
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void merge_sequence(const Params& p, int T, int b, int P, int nt, int nthreads)
+{
+    const int G = p.num_ctas;
+    // which blocks hold the parts follows from the schedule alone
+    const int i_first = cta_of_tile(P, T, G), last_cta = cta_of_tile((long long)P + nt - 1, T, G);
+    const int first_slot = ((long long)P == span_begin(i_first, T, G)) ? 2 * i_first : 2 * i_first + 1;
+    merge_parts<D, 6, 1>(p, T, b, i_first, first_slot, last_cta, nthreads);
+    if (threadIdx.x == 0) ws_arrivals(p.workspace, p.B)[b] = 0;   // ready for the next call
+}
+
 template <int D, int HP>
 struct TcLayout {
     static constexpr int HG = HP / kHeadsPerThread;          // head groups = softmax warpgroups
@@ -296,6 +381,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         mbar_init(&bars.p_full, L::kSoftmaxThreads); mbar_init(&bars.p_empty, 1);
         mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, L::kSoftmaxThreads);
         misc.abort_flag = 0;
+        misc.n_pending = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -312,6 +398,13 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         ws_header(p.workspace)[kHdrNumCtas] = G;
     }
     const int N = (T > 0) ? (int)(span_begin(cta + 1, T, G) - span_begin(cta, T, G)) : 0;   // tiles of this block
+    // Empty sequences own no tile: their output rows are zeroed here, round-robin over the blocks.
+    for (int b = cta; b < p.B; b += G) {
+        if (clamp_len(p.lengths[b], p.Lmax) == 0) {
+            float4* dst = reinterpret_cast<float4*>(p.out + (size_t)b * H * D);
+            for (int i = tid; i < H * D / 4; i += L::kThreads) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
 
     if (N > 0) {
         if (warp == 0) {
@@ -566,6 +659,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 const bool whole = c.w.seg_is_whole();
                 const bool use_lo = c.w.len <= p.lo_max_len;
                 const int slot_id = c.w.seg_slot(cta);
+                const long long c_P = c.w.P;
+                const int c_nt = c.w.nt;
                 if (c.w.seg_owns_first_tile() && sid == 0) {
                     SeqInfo si;
                     si.first_slot = whole ? -1 : slot_id;
@@ -758,6 +853,22 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                             if (hb + i < H) dst[(size_t)i * D] = o[j][i];
                     }
                 }
+                if (!whole) {
+                    // Publish this partial result.  The block that delivers a sequence's last partial result
+                    // merges all of them after its own tiles are done (merge_sequence below).
+                    __threadfence();
+                    softmax_bar_sync(NSM);
+                    if (sid == 0) {
+                        const int i_first = cta_of_tile(c_P, T, G), i_last = cta_of_tile(c_P + c_nt - 1, T, G);
+                        const int nparts = (T >= G) ? (i_last - i_first + 1) : c_nt;   // T < G: one tile per block
+                        const int old = atomicAdd(ws_arrivals(p.workspace, p.B) + b, 1);
+                        if (old == nparts - 1) {
+                            __threadfence();
+                            const int k = misc.n_pending++;
+                            misc.pending[k] = b; misc.pending_p[k] = (int)c_P; misc.pending_nt[k] = c_nt;
+                        }
+                    }
+                }
                 softmax_bar_sync(NSM);     // misc.m / misc.alpha are rewritten by the next segment
                 PROF_END(kProfSmEpilogue);
                 }
@@ -768,6 +879,15 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 
     __syncwarp();
     __syncthreads();
+    if (!misc.abort_flag) {
+        const int n_pending = misc.n_pending;
+#ifndef MQA_X_SKIP_MERGE
+        for (int k = 0; k < n_pending; ++k)
+            merge_sequence<D>(p, T, misc.pending[k], misc.pending_p[k], misc.pending_nt[k], L::kThreads);
+#else
+        if (tid == 0) for (int k = 0; k < n_pending; ++k) ws_arrivals(p.workspace, p.B)[misc.pending[k]] = 0;
+#endif
+    }
 #ifdef MQA_TC_PROFILE
     if (tid == 0) {
         unsigned long long ns1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
@@ -828,27 +948,48 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t dim0, uint64_t dim1
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Host-side caches: the shared-memory limit and the kernel attribute are per device; the three tensor
+// maps depend only on (pointers, shape) and are reused while a caller keeps decoding from the same buffers.
+constexpr int kMaxDevices = 64;
+
+struct MapCache {
+    const void *q = nullptr, *k = nullptr, *v = nullptr;
+    int B = 0, H = 0, D = 0, Lmax = 0, hp = 0;
+    CUtensorMap mq, mk, mv;
+};
+
 template <int D, int HP>
 cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
 {
+    using L = TcLayout<D, HP>;
     Params p = p_in;
     p.lo_max_len = lo_max_len_setting();
-    using L = TcLayout<D, HP>;
-    int dev = 0, smem_limit = 0;
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (e != cudaSuccess) return e;
-    const int nslots = L::slots_for(smem_limit);
-    if (nslots < kMinSlots) return cudaErrorInvalidConfiguration;
-    const int smem = L::smem_bytes(nslots);
-    CUtensorMap mq, mk, mv;
-    if (!encode_map(&mq, p.q, p.D, p.H, p.B, HP) || !encode_map(&mk, p.k, p.D, p.Lmax, p.B, 128) ||
-        !encode_map(&mv, p.v, p.D, p.Lmax, p.B, 64))
-        return cudaErrorInvalidValue;
-    e = cudaFuncSetAttribute(mqa_tc_kernel<D, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    mqa_tc_kernel<D, HP><<<p.num_ctas, L::kThreads, smem, stream>>>(p, mq, mk, mv, nslots);
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    static int s_nslots[kMaxDevices] = {};      // 0 = not yet configured on that device
+    int nslots = s_nslots[dev];
+    if (nslots == 0) {
+        int smem_limit = 0;
+        e = cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        if (e != cudaSuccess) return e;
+        nslots = L::slots_for(smem_limit);
+        if (nslots < kMinSlots) return cudaErrorInvalidConfiguration;
+        e = cudaFuncSetAttribute(mqa_tc_kernel<D, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::smem_bytes(nslots));
+        if (e != cudaSuccess) return e;
+        s_nslots[dev] = nslots;
+    }
+    thread_local MapCache mc;
+    if (mc.q != p.q || mc.k != p.k || mc.v != p.v || mc.B != p.B || mc.H != p.H || mc.D != p.D || mc.Lmax != p.Lmax || mc.hp != HP) {
+        if (!encode_map(&mc.mq, p.q, p.D, p.H, p.B, HP) || !encode_map(&mc.mk, p.k, p.D, p.Lmax, p.B, 128) ||
+            !encode_map(&mc.mv, p.v, p.D, p.Lmax, p.B, 64)) {
+            mc.q = nullptr;
+            return cudaErrorInvalidValue;
+        }
+        mc.q = p.q; mc.k = p.k; mc.v = p.v; mc.B = p.B; mc.H = p.H; mc.D = p.D; mc.Lmax = p.Lmax; mc.hp = HP;
+    }
+    mqa_tc_kernel<D, HP><<<p.num_ctas, L::kThreads, L::smem_bytes(nslots), stream>>>(p, mc.mq, mc.mk, mc.mv, nslots);
     return cudaGetLastError();
 }
 

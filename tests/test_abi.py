@@ -44,9 +44,9 @@ def test_workspace_bytes(L):
     assert binding.mqa_decode_workspace_bytes(2, 65, 64, 128) == 0     # H > 64
     n = binding.mqa_decode_workspace_bytes(2, 4, 64, 128)
     slot = (2 * 4 + 4 * 64) * 4
-    assert n == 256 + 256 + 2 * binding.MQA_MAX_CTAS * slot
+    assert n == 256 + 256 + 256 + 2 * binding.MQA_MAX_CTAS * slot
     big = binding.mqa_decode_workspace_bytes(512, 48, 256, 2048)
-    assert big == 256 + 4096 + 2 * binding.MQA_MAX_CTAS * (2 * 48 + 48 * 256) * 4
+    assert big == 256 + 4096 + 2048 + 2 * binding.MQA_MAX_CTAS * (2 * 48 + 48 * 256) * 4
     assert binding.mqa_decode_host_scratch_bytes(2, 4, 64, 128) > n
 
 

@@ -58,4 +58,4 @@ def test_static_workspace_rejects_what_does_not_fit():
     rc = binding.lib().mqa_decode_static(0x1000, 0x2000, 0x3000, 0x4000, 0x5000,
                                          3_000_000, 1, 64, 1, 1.0, None)
     assert rc == binding.MQA_ERR_WORKSPACE_TOO_SMALL
-    assert 256 + 8 * 3_000_000 > binding.MQA_STATIC_WORKSPACE_BYTES
+    assert 256 + 12 * 3_000_000 > binding.MQA_STATIC_WORKSPACE_BYTES
