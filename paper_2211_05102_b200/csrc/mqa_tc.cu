@@ -132,14 +132,6 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
         : "memory");
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate, issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
 // Arrive on an mbarrier once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(void* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -202,18 +194,30 @@ __device__ __forceinline__ bool softmax_bar_or(bool flag, int nthreads) {
 }
 __device__ __forceinline__ void softmax_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
-// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle = 2 at bits 61..63).
-// K-major operand, rows of 128 B (64 bf16), 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+// Shared-memory matrix descriptors (sm_100 format), split into a constant high word (8-row groups 1024 B
+// apart, version 1, 128-byte swizzle) and a 32-bit low word (start address >> 4, leading offset >> 4), so
+// that stepping through an operand is one 32-bit add: shared-memory addresses stay below 256 KB and never
+// carry out of the 14-bit address field.
+//   K-major operand: rows of 128 B (64 bf16); the leading offset is unused.
+//   MN-major operand: 64 contiguous MN elements per 128-B row, the next 64 MN elements
+//   `mn_group_bytes` further on.
+// D[tmem] (+)= A * B with bf16 inputs and fp32 accumulation, issued by one thread.
+constexpr uint32_t kDescHiSw128 = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // SBO, version, 128-byte swizzle
+__device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t saddr, uint32_t mn_group_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((mn_group_bytes >> 4) << 16);
 }
-// MN-major operand: 64 contiguous MN elements per row of 128 B, the next 64 MN elements
-// `mn_group_bytes` further on, 8-row K groups 1024 B apart.
-__device__ __forceinline__ uint64_t desc_mnmajor_sw128(uint32_t saddr, uint32_t mn_group_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_group_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(ACCUMULATE ? 1 : 0) : "memory");
 }
+
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; *_mn_major selects a transposed operand.
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn_major, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
@@ -243,9 +247,31 @@ struct TileCursor {
     }
 };
 
+// Lean walk over the tiles of a block's run for the MMA issuer: everything it needs per tile is a
+// couple of int compares; the 64-bit schedule arithmetic runs once per segment.
+struct SegIter {
+    SegmentWalker w;
+    int seg, ti, nt_seg, len;
+    bool valid;
+    __device__ void load() { ti = 0; nt_seg = w.seg_t1() - w.seg_t0(); len = w.len; }
+    __device__ void init(const Params& p, int T, int cta, const SchedShared& sh) {
+        w.init(p.lengths, p.B, p.Lmax, kTileShift, T, p.num_ctas, cta, sh.b0, sh.p0);
+        seg = 0; valid = !w.done();
+        if (valid) load();
+    }
+    __device__ bool first() const { return ti == 0; }
+    __device__ bool last() const { return ti + 1 == nt_seg; }
+    __device__ void next() {
+        if (++ti == nt_seg) {
+            w.next(); ++seg;
+            valid = !w.done();
+            if (valid) load();
+        }
+    }
+};
+
 // Ring bookkeeping: the producer and both consumers enumerate load items in the same order
 // K(0), K(1), V(0), K(2), V(1), ..., K(N-1), V(N-2), V(N-1); every item fills SPT consecutive slots.
-__device__ __forceinline__ int item_of_k(int n) { return n == 0 ? 0 : 2 * n - 1; }
 __device__ __forceinline__ int item_of_v(int n, int N) { return n == N - 1 ? 2 * N - 1 : 2 * n + 2; }
 
 // Log-sum-exp merge of the partial results of one cut sequence, by every thread of the block:
@@ -376,10 +402,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars.q_full[i], 1); mbar_init(&bars.q_empty[i], 1);
-            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads);
+            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32);
         }
-        mbar_init(&bars.p_full, L::kSoftmaxThreads); mbar_init(&bars.p_empty, 1);
-        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, L::kSoftmaxThreads);
+        mbar_init(&bars.p_full, L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty, 1);
+        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, L::kSoftmaxThreads / 32);
         misc.abort_flag = 0;
         misc.n_pending = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -434,27 +460,36 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     __syncwarp();
                 }
 #endif
+                // The SPT chunk loads of one K tile cover the same DRAM rows (each takes 128 of every 512 bytes),
+                // so they are issued back to back once all their slots are free.
+                {
+                    int sl = pslot; uint32_t ph = pphase;
 #pragma unroll
-                for (int ch = 0; ch < SPT; ++ch) {
-                    const int slot = pslot;
-                    {
+                    for (int ch = 0; ch < SPT; ++ch) {
                         PROF_BEGIN();
-                        if (!mbar_wait(&bars.empty[slot], pphase ^ 1, abort_flag)) { ok = false; return; }
+                        if (!mbar_wait(&bars.empty[sl], ph ^ 1, abort_flag)) { ok = false; return; }
                         PROF_END(kProfProdEmpty);
+                        if (++sl == nslots) { sl = 0; ph ^= 1; }
                     }
-                    TRACE(0, 1, slot_seq);
-                    if (elect_one_sync()) {
-#ifdef MQA_X_NOLOAD
-                        mbar_arrive(&bars.full[slot]);
-#else
-                        mbar_expect_tx(&bars.full[slot], kSlotBytes);
-                        tma_load_3d(ring + (size_t)slot * kSlotBytes, &map_k, &bars.full[slot], ch * 64, c.row0(), c.w.b, policy);
-#endif
-                    }
-                    __syncwarp();
-                    ++slot_seq;
-                    if (++pslot == nslots) { pslot = 0; pphase ^= 1; }
                 }
+                if (elect_one_sync()) {
+                    int sl = pslot;
+#pragma unroll
+                    for (int ch = 0; ch < SPT; ++ch) {
+#ifdef MQA_X_NOLOAD
+                        mbar_arrive(&bars.full[sl]);
+#else
+                        mbar_expect_tx(&bars.full[sl], kSlotBytes);
+                        tma_load_3d(ring + (size_t)sl * kSlotBytes, &map_k, &bars.full[sl], ch * 64, c.row0(), c.w.b, policy);
+#endif
+                        if (++sl == nslots) sl = 0;
+                    }
+                }
+                __syncwarp();
+                TRACE(0, 1, slot_seq);
+                slot_seq += SPT;
+                pslot += SPT;
+                if (pslot >= nslots) { pslot -= nslots; pphase ^= 1; }
             };
             auto load_v = [&](const TileCursor& c) {
 #pragma unroll
@@ -498,36 +533,39 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             }
         } else if (warp == 1) {
             // =============================== MMA issuer (whole warp waits, one lane issues) ===============================
+            // This warp's own instruction stream is the critical resource (48 MMAs and ~20 barrier operations per
+            // tile, issued by one thread), so it walks the schedule with plain counters, keeps every descriptor as a
+            // constant high word plus a 32-bit low word, and hard-codes the accumulate flag.
             constexpr uint32_t idesc_qk = make_idesc(HP, false, false);
             constexpr uint32_t idesc_pv = make_idesc(HP, true, true);
-            TileCursor ck, cv;
-            ck.init(p, T, cta, misc.sched);
-            cv = ck;
+            SegIter iq, iv;            // QK runs one tile ahead of PV
+            iq.init(p, T, cta, misc.sched);
+            iv = iq;
             int nq = 0, np = 0;
             int cslot = 0;             // ring slot consumed next: slots are used in the order they were filled
             uint32_t cphase = 0;
             bool ok = true;
             int trace_n = 0; (void)trace_n;
-            const uint32_t q_addr = smem_u32(q_buf);
-            const uint64_t desc_ring0 = desc_kmajor_sw128(smem_u32(ring));
-            const uint64_t desc_ring0_mn = desc_mnmajor_sw128(smem_u32(ring), 8192);
-            const uint64_t desc_phi = desc_mnmajor_sw128(smem_u32(p_hi), 8192);
-            const uint64_t desc_plo = desc_mnmajor_sw128(smem_u32(p_lo), 8192);
+            const uint32_t q_lo = desc_lo_kmajor(smem_u32(q_buf));
+            const uint32_t ring_lo_k = desc_lo_kmajor(smem_u32(ring));
+            const uint32_t ring_lo_mn = desc_lo_mnmajor(smem_u32(ring), 8192);
+            const uint32_t phi_lo = desc_lo_mnmajor(smem_u32(p_hi), 8192);
+            const uint32_t plo_lo = desc_lo_mnmajor(smem_u32(p_lo), 8192);
             PROF_BEGIN();
-            auto issue_qk = [&](const TileCursor& c) {
+            auto issue_qk = [&]() {
                 const int sb = nq & 1;
                 { PROF_BEGIN();
                   if (!mbar_wait(&bars.s_empty[sb], ((nq >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
                   PROF_END(kProfMmaSEmpty); }
-                const int qb = c.seg & 1;
-                if (c.first_in_seg()) {
+                const int qb = iq.seg & 1;
+                if (iq.first()) {
                     PROF_BEGIN();
-                    if (!mbar_wait(&bars.q_full[qb], (c.seg >> 1) & 1, abort_flag)) { ok = false; return; }
+                    if (!mbar_wait(&bars.q_full[qb], (iq.seg >> 1) & 1, abort_flag)) { ok = false; return; }
                     PROF_END(kProfMmaQFull);
                 }
                 const uint32_t d_tmem = tmem + (uint32_t)(sb * 64);
-                const uint64_t db0 = desc_kmajor_sw128(q_addr + (uint32_t)(qb * L::kQBytes));
-                const bool last = c.last_in_seg();
+                const uint32_t qlo = q_lo + (uint32_t)(qb * (L::kQBytes >> 4));
+                const bool last = iq.last();
                 TRACE(1, 10, nq);   // QK: s_empty and q ready
 #pragma unroll
                 for (int ch = 0; ch < SPT; ++ch) {
@@ -538,13 +576,15 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
                     tc_fence_after();
                     TRACE(1, 11 + ch, nq);   // K chunk landed
-                    const uint64_t da = desc_ring0 + (uint64_t)((uint32_t)slot * (kSlotBytes >> 4));
-                    const uint64_t db = db0 + (uint64_t)(ch * (HP * 128 >> 4));
+                    const uint32_t alo = ring_lo_k + (uint32_t)slot * (kSlotBytes >> 4);
+                    const uint32_t blo = qlo + (uint32_t)(ch * (HP * 128 >> 4));
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_QK
+                        if (ch == 0) umma_bf16_lo<false>(d_tmem, alo, blo, kDescHiSw128, idesc_qk);
+                        else         umma_bf16_lo<true>(d_tmem, alo, blo, kDescHiSw128, idesc_qk);
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
-                            umma_bf16(d_tmem, da + (uint64_t)(ks * 2), db + (uint64_t)(ks * 2), idesc_qk, (ch | ks) ? 1u : 0u);
+                        for (int ks = 1; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
+                            umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * 2), blo + (uint32_t)(ks * 2), kDescHiSw128, idesc_qk);
 #endif
                         umma_commit(&bars.empty[slot]);
                         if (ch == SPT - 1) {
@@ -556,22 +596,25 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 }
                 TRACE(1, 15, nq);   // QK issued
                 ++nq;
+                iq.next();
             };
-            auto issue_pv = [&](const TileCursor& c, bool use_lo) {
+            auto issue_pv = [&]() {
                 { PROF_BEGIN();
                   if (!mbar_wait(&bars.p_full, np & 1, abort_flag)) { ok = false; return; }
                   PROF_END(kProfMmaPFull); }
-                if (c.first_in_seg()) {
+                const bool fresh = iv.first();
+                if (fresh) {
                     PROF_BEGIN();
-                    if (!mbar_wait(&bars.o_empty, (c.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
+                    if (!mbar_wait(&bars.o_empty, (iv.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
                     PROF_END(kProfMmaOEmpty);
                 }
                 tc_fence_after();
                 TRACE(1, 20, np);   // P ready
-                const bool fresh = c.first_in_seg();
-                const bool last = c.last_in_seg();
+                const bool last = iv.last();
+                const bool use_lo = iv.len <= p.lo_max_len;
 #pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
+                    constexpr int kStep = 2048 >> 4;               // 16 cache rows of 128 B
                     const int r = vi / NACC, j = vi % NACC;
                     const int slot = cslot;
                     { PROF_BEGIN();
@@ -581,17 +624,21 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     tc_fence_after();
                     TRACE(1, 21 + vi, np);   // V slot landed
                     const uint32_t d_tmem = tmem + 128u + (uint32_t)(j * 64);
-                    const uint64_t da = desc_ring0_mn + (uint64_t)((uint32_t)slot * (kSlotBytes >> 4));
-                    const uint64_t dbh = desc_phi + (uint64_t)(r * (64 * 128 >> 4));
-                    const uint64_t dbl = desc_plo + (uint64_t)(r * (64 * 128 >> 4));
+                    const uint32_t alo = ring_lo_mn + (uint32_t)slot * (kSlotBytes >> 4);
+                    const uint32_t bhl = phi_lo + (uint32_t)(r * (64 * 128 >> 4));
+                    const uint32_t bll = plo_lo + (uint32_t)(r * (64 * 128 >> 4));
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_PV
+                        // the first MMA of a segment's accumulator overwrites it
+                        if (r == 0 && fresh) umma_bf16_lo<false>(d_tmem, alo, bhl, kDescHiSw128, idesc_pv);
+                        else                 umma_bf16_lo<true>(d_tmem, alo, bhl, kDescHiSw128, idesc_pv);
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {   // 4 x 16 cache rows per 64-row slot
-                            const uint32_t acc = (fresh && r == 0 && ks == 0) ? 0u : 1u;
-                            umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbh + (uint64_t)(ks * (2048 >> 4)), idesc_pv, acc);
-                            if (use_lo)
-                                umma_bf16(d_tmem, da + (uint64_t)(ks * (2048 >> 4)), dbl + (uint64_t)(ks * (2048 >> 4)), idesc_pv, 1u);
+                        for (int ks = 1; ks < 4; ++ks)             // 4 x 16 cache rows per 64-row slot
+                            umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * kStep), bhl + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
+                        if (use_lo) {
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * kStep), bll + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
                         }
 #endif
                         umma_commit(&bars.empty[slot]);
@@ -604,6 +651,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 }
                 TRACE(1, 25, np);   // PV issued
                 ++np;
+                iv.next();
             };
 #ifdef MQA_X_LOADONLY
             // experiment: free every slot as soon as it has landed (measures the staging rate alone)
@@ -614,10 +662,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 __syncwarp();
             }
 #else
-            issue_qk(ck); ck.advance();
-            while (ok && cv.valid()) {
-                if (ck.valid()) { issue_qk(ck); ck.advance(); }
-                if (ok) { issue_pv(cv, cv.w.len <= p.lo_max_len); cv.advance(); }
+            issue_qk();
+            while (ok && iv.valid) {
+                if (iq.valid) issue_qk();
+                if (ok) issue_pv();
             }
 #endif
             PROF_END(kProfMmaTotal);
@@ -685,7 +733,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     tmem_ld16(lane_base + (uint32_t)(sb * 64 + hb), y);
                     tmem_wait_ld();
                     tc_fence_before();
-                    mbar_arrive(&bars.s_empty[sb]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.s_empty[sb]);   // one arrival per warp
                     const bool valid = row < nvalid;
                     // y = scale_log2 * logit (-inf for rows beyond the sequence); does any y exceed m + threshold?
                     float xmax = -INFINITY;
@@ -799,7 +848,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         if (!ok) break;
                     }
                     fence_proxy_async();
-                    mbar_arrive(&bars.p_full);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.p_full);
                     TRACE(2, 34, ns);   // P published
                     first = false;
                     ++ns;
@@ -837,7 +887,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 for (int j = 0; j < NACC; ++j) tmem_ld16(lane_base + 128u + (uint32_t)(j * 64 + hb), o[j]);
                 tmem_wait_ld();
                 tc_fence_before();
-                mbar_arrive(&bars.o_empty);      // the accumulators are in registers: the next segment may overwrite them
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.o_empty);   // the accumulators are in registers: the next segment may overwrite them
 #pragma unroll
                 for (int j = 0; j < NACC; ++j) {
                     const int d = j * 128 + row;
