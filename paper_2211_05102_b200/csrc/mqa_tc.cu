@@ -32,19 +32,28 @@ constexpr int kTileShift = 7;
 constexpr int kTileRows = 128;
 constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 64 rows x 128 cols (V)
 constexpr int kMaxSlots = 12;
-constexpr int kMinSlots = 8;
+constexpr int kMinSlots = 4;               // any depth >= 1 is deadlock-free (slots are filled and drained in one order)
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logit units: rescale only when a logit exceeds m + 8
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds; only a deadlock gets here
 constexpr int kSoftmaxWarp0 = 4;
-constexpr uint32_t kTmemCols = 256;        // S0 @0, S1 @64, O0 @128, O1 @192
+constexpr uint32_t kTmemCols = 512;        // 4 S buffers @0,64,128,192; accumulator set s (segment parity) @256+128s, its D half j @+64j
+#ifndef MQA_QK_LEAD
+#define MQA_QK_LEAD 1
+#endif
+#ifndef MQA_P_BUFS
+#define MQA_P_BUFS 1
+#endif
+constexpr int kPBufs = MQA_P_BUFS;         // probability buffers (each hi + lo)
+constexpr int kQkLead = MQA_QK_LEAD;                 // the logits of tile t+2 are issued before the weighted values of tile t
+constexpr uint32_t kOCol = 256;
 
 struct Barriers {
     unsigned long long full[kMaxSlots];
     unsigned long long empty[kMaxSlots];
     unsigned long long q_full[2], q_empty[2];
-    unsigned long long s_full[2], s_empty[2];
-    unsigned long long p_full, p_empty;
-    unsigned long long o_full, o_empty;
+    unsigned long long s_full[4], s_empty[4];
+    unsigned long long p_full[2], p_empty[2];
+    unsigned long long o_full[2], o_empty[2];
 };
 
 struct Misc {
@@ -57,7 +66,8 @@ struct Misc {
     int pending_p[2], pending_nt[2];   // first global tile and tile count of those sequences
     float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
     __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
-    __align__(16) float alpha[kMaxHeads];  // rescale factors; row sums in the epilogue
+    __align__(16) float alpha[kMaxHeads];  // rescale factors
+    __align__(16) float lsum[2][kMaxHeads]; // row sums of a finished segment, by segment parity, until its epilogue has run
 };
 
 // Optional cycle accounting (compile with -DMQA_TC_PROFILE): block 0 adds the cycles each role
@@ -84,7 +94,7 @@ struct Misc {
 #endif
 enum { kProfProdEmpty = 0, kProfMmaSEmpty, kProfMmaQFull, kProfMmaKFull, kProfMmaPFull, kProfMmaOEmpty, kProfMmaVFull,
        kProfSmSFull, kProfSmBar, kProfSmPEmpty, kProfSmRescale, kProfSmStore, kProfSmEpilogue, kProfSmTotal, kProfMmaTotal,
-       kProfProdTotal, kProfSmLoad, kProfSmOFull };
+       kProfProdTotal, kProfSmLoad, kProfSmOFull, kProfSmScale, kProfSmPublish };
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -251,9 +261,10 @@ struct TileCursor {
 // couple of int compares; the 64-bit schedule arithmetic runs once per segment.
 struct SegIter {
     SegmentWalker w;
-    int seg, ti, nt_seg, len;
+    int seg, ti, nt_seg, len, t0;
     bool valid;
-    __device__ void load() { ti = 0; nt_seg = w.seg_t1() - w.seg_t0(); len = w.len; }
+    __device__ void load() { ti = 0; t0 = w.seg_t0(); nt_seg = w.seg_t1() - t0; len = w.len; }
+    __device__ int nvalid() const { return min(kTileRows, len - ((t0 + ti) << kTileShift)); }   // valid rows of the current tile
     __device__ void init(const Params& p, int T, int cta, const SchedShared& sh) {
         w.init(p.lengths, p.B, p.Lmax, kTileShift, T, p.num_ctas, cta, sh.b0, sh.p0);
         seg = 0; valid = !w.done();
@@ -271,8 +282,8 @@ struct SegIter {
 };
 
 // Ring bookkeeping: the producer and both consumers enumerate load items in the same order
-// K(0), K(1), V(0), K(2), V(1), ..., K(N-1), V(N-2), V(N-1); every item fills SPT consecutive slots.
-__device__ __forceinline__ int item_of_v(int n, int N) { return n == N - 1 ? 2 * N - 1 : 2 * n + 2; }
+// K(0), .., K(lead), V(0), K(lead+1), V(1), ..., K(N-1), V(N-1-lead), .., V(N-1) with lead = kQkLead; every item fills
+// SPT consecutive slots.
 
 // Log-sum-exp merge of the partial results of one cut sequence, by every thread of the block:
 //   M = max_s m_s;  out = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s
@@ -365,7 +376,7 @@ struct TcLayout {
     static constexpr int NACC = D / 128;          // 128-wide halves of D = output accumulators
     static constexpr int kQBytes = HP * D * 2;    // one q buffer: D/64 chunks of [HP rows x 128 B]
     static constexpr int kPBytes = 128 * 128;     // one probability buffer: 128 cache rows x 128 B (up to 64 heads)
-    static constexpr int kFixed = 2 * kQBytes + 2 * kPBytes + (int)sizeof(Misc);
+    static constexpr int kFixed = 2 * kQBytes + 2 * kPBufs * kPBytes + (int)sizeof(Misc);   // q x2, (hi, lo) x kPBufs
     static int slots_for(int smem_limit) {
         int n = (smem_limit - 1024 - kFixed) / kSlotBytes;
         return n > kMaxSlots ? kMaxSlots : n;
@@ -384,9 +395,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* ring = smem;
     unsigned char* q_buf = ring + (size_t)nslots * kSlotBytes;       // 2 buffers
-    unsigned char* p_hi = q_buf + 2 * L::kQBytes;
-    unsigned char* p_lo = p_hi + L::kPBytes;
-    Misc& misc = *reinterpret_cast<Misc*>(p_lo + L::kPBytes);
+    unsigned char* p_buf = q_buf + 2 * L::kQBytes;                   // 2 buffers of (hi, lo)
+    Misc& misc = *reinterpret_cast<Misc*>(p_buf + 2 * kPBufs * L::kPBytes);
     Barriers& bars = misc.bars;
     volatile int* abort_flag = &misc.abort_flag;
 
@@ -402,10 +412,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars.q_full[i], 1); mbar_init(&bars.q_empty[i], 1);
-            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32);
         }
-        mbar_init(&bars.p_full, L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty, 1);
-        mbar_init(&bars.o_full, 1); mbar_init(&bars.o_empty, L::kSoftmaxThreads / 32);
+        for (int i = 0; i < 4; ++i) { mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars.p_full[i], L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], L::kSoftmaxThreads / 32); }
         misc.abort_flag = 0;
         misc.n_pending = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -466,9 +476,11 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     int sl = pslot; uint32_t ph = pphase;
 #pragma unroll
                     for (int ch = 0; ch < SPT; ++ch) {
+#ifndef MQA_X_NOCHUNKSYNC
                         PROF_BEGIN();
                         if (!mbar_wait(&bars.empty[sl], ph ^ 1, abort_flag)) { ok = false; return; }
                         PROF_END(kProfProdEmpty);
+#endif
                         if (++sl == nslots) { sl = 0; ph ^= 1; }
                     }
                 }
@@ -476,7 +488,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     int sl = pslot;
 #pragma unroll
                     for (int ch = 0; ch < SPT; ++ch) {
-#ifdef MQA_X_NOLOAD
+#if defined(MQA_X_NOCHUNKSYNC)
+#elif defined(MQA_X_NOLOAD)
                         mbar_arrive(&bars.full[sl]);
 #else
                         mbar_expect_tx(&bars.full[sl], kSlotBytes);
@@ -496,15 +509,19 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 for (int vi = 0; vi < SPT; ++vi) {
                     const int r = vi / NACC, j = vi % NACC;
                     const int slot = pslot;
+#ifndef MQA_X_NOCHUNKSYNC
                     {
                         PROF_BEGIN();
                         if (!mbar_wait(&bars.empty[slot], pphase ^ 1, abort_flag)) { ok = false; return; }
                         PROF_END(kProfProdEmpty);
                     }
+#endif
                     TRACE(0, 2, slot_seq);
                     if (elect_one_sync()) {
                         unsigned char* dst = ring + (size_t)slot * kSlotBytes;
-#ifdef MQA_X_NOLOAD
+#if defined(MQA_X_NOCHUNKSYNC)
+                        (void)dst;
+#elif defined(MQA_X_NOLOAD)
                         (void)dst; mbar_arrive(&bars.full[slot]);
 #else
                         mbar_expect_tx(&bars.full[slot], kSlotBytes);
@@ -517,10 +534,9 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     if (++pslot == nslots) { pslot = 0; pphase ^= 1; }
                 }
             };
-            load_k(ck); ck.advance();
-            while (ok && cv.valid()) {
-                if (ck.valid()) { load_k(ck); ck.advance(); }
-                if (ok) { load_v(cv); cv.advance(); }
+            for (int n = 0; ok && n < N + kQkLead; ++n) {
+                if (n < N) { load_k(ck); ck.advance(); }
+                if (ok && n >= kQkLead) { load_v(cv); cv.advance(); }
             }
             PROF_END(kProfProdTotal);
             if (!ok) {
@@ -549,13 +565,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(q_buf));
             const uint32_t ring_lo_k = desc_lo_kmajor(smem_u32(ring));
             const uint32_t ring_lo_mn = desc_lo_mnmajor(smem_u32(ring), 8192);
-            const uint32_t phi_lo = desc_lo_mnmajor(smem_u32(p_hi), 8192);
-            const uint32_t plo_lo = desc_lo_mnmajor(smem_u32(p_lo), 8192);
+            const uint32_t p_lo32 = desc_lo_mnmajor(smem_u32(p_buf), 8192);
             PROF_BEGIN();
             auto issue_qk = [&]() {
-                const int sb = nq & 1;
+                const int sb = nq & 3;
                 { PROF_BEGIN();
-                  if (!mbar_wait(&bars.s_empty[sb], ((nq >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
+                  if (!mbar_wait(&bars.s_empty[sb], ((nq >> 2) & 1) ^ 1, abort_flag)) { ok = false; return; }
                   PROF_END(kProfMmaSEmpty); }
                 const int qb = iq.seg & 1;
                 if (iq.first()) {
@@ -570,9 +585,11 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 #pragma unroll
                 for (int ch = 0; ch < SPT; ++ch) {
                     const int slot = cslot;
+#ifndef MQA_X_NOCHUNKSYNC
                     { PROF_BEGIN();
                       if (!mbar_wait(&bars.full[slot], cphase, abort_flag)) { ok = false; return; }
                       PROF_END(kProfMmaKFull); }
+#endif
                     if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
                     tc_fence_after();
                     TRACE(1, 11 + ch, nq);   // K chunk landed
@@ -586,13 +603,16 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         for (int ks = 1; ks < 4; ++ks)   // 4 x 16 columns of D per 64-column chunk
                             umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * 2), blo + (uint32_t)(ks * 2), kDescHiSw128, idesc_qk);
 #endif
+#ifndef MQA_X_NOCHUNKSYNC
                         umma_commit(&bars.empty[slot]);
+#endif
                         if (ch == SPT - 1) {
                             umma_commit(&bars.s_full[sb]);
                             if (last) umma_commit(&bars.q_empty[qb]);
                         }
                     }
                     __syncwarp();
+
                 }
                 TRACE(1, 15, nq);   // QK issued
                 ++nq;
@@ -600,33 +620,49 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             };
             auto issue_pv = [&]() {
                 { PROF_BEGIN();
-                  if (!mbar_wait(&bars.p_full, np & 1, abort_flag)) { ok = false; return; }
+                  if (!mbar_wait(&bars.p_full[np % kPBufs], (np / kPBufs) & 1, abort_flag)) { ok = false; return; }
                   PROF_END(kProfMmaPFull); }
                 const bool fresh = iv.first();
                 if (fresh) {
                     PROF_BEGIN();
-                    if (!mbar_wait(&bars.o_empty, (iv.seg & 1) ^ 1, abort_flag)) { ok = false; return; }
+                    if (!mbar_wait(&bars.o_empty[iv.seg & 1], ((iv.seg >> 1) & 1) ^ 1, abort_flag)) { ok = false; return; }
                     PROF_END(kProfMmaOEmpty);
                 }
                 tc_fence_after();
                 TRACE(1, 20, np);   // P ready
                 const bool last = iv.last();
                 const bool use_lo = iv.len <= p.lo_max_len;
+                const int nvalid = iv.nvalid();
 #pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
                     constexpr int kStep = 2048 >> 4;               // 16 cache rows of 128 B
                     const int r = vi / NACC, j = vi % NACC;
                     const int slot = cslot;
+#ifndef MQA_X_NOCHUNKSYNC
                     { PROF_BEGIN();
                       if (!mbar_wait(&bars.full[slot], cphase, abort_flag)) { ok = false; return; }
                       PROF_END(kProfMmaVFull); }
+#endif
                     if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
+                    if (nvalid < kTileRows) {
+                        // Rows beyond the sequence may hold any bits (0 * NaN would poison the accumulator): zero them
+                        // in the staged tile.  This warp consumes the ring strictly in order, so the slot is known to
+                        // hold this tile.
+                        for (int lr = max(0, nvalid - r * 64) + lane; lr < 64; lr += 32) {
+                            uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + lr * 128);
+                            uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + lr * 128);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) { dst0[i] = make_uint4(0, 0, 0, 0); dst1[i] = make_uint4(0, 0, 0, 0); }
+                        }
+                        fence_proxy_async();
+                        __syncwarp();
+                    }
                     tc_fence_after();
                     TRACE(1, 21 + vi, np);   // V slot landed
-                    const uint32_t d_tmem = tmem + 128u + (uint32_t)(j * 64);
+                    const uint32_t d_tmem = tmem + kOCol + (uint32_t)((iv.seg & 1) * 128 + j * 64);
                     const uint32_t alo = ring_lo_mn + (uint32_t)slot * (kSlotBytes >> 4);
-                    const uint32_t bhl = phi_lo + (uint32_t)(r * (64 * 128 >> 4));
-                    const uint32_t bll = plo_lo + (uint32_t)(r * (64 * 128 >> 4));
+                    const uint32_t bhl = p_lo32 + (uint32_t)(((np % kPBufs) * 2 * L::kPBytes + r * 64 * 128) >> 4);
+                    const uint32_t bll = bhl + (uint32_t)(L::kPBytes >> 4);
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_PV
                         // the first MMA of a segment's accumulator overwrites it
@@ -641,10 +677,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                                 umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * kStep), bll + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
                         }
 #endif
+#ifndef MQA_X_NOCHUNKSYNC
                         umma_commit(&bars.empty[slot]);
+#endif
                         if (vi == SPT - 1) {
-                            umma_commit(&bars.p_empty);
-                            if (last) umma_commit(&bars.o_full);
+                            umma_commit(&bars.p_empty[np % kPBufs]);
+                            if (last) umma_commit(&bars.o_full[iv.seg & 1]);
                         }
                     }
                     __syncwarp();
@@ -662,10 +700,9 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 __syncwarp();
             }
 #else
-            issue_qk();
-            while (ok && iv.valid) {
-                if (iq.valid) issue_qk();
-                if (ok) issue_pv();
+            for (int n = 0; ok && n < N + kQkLead; ++n) {
+                if (n < N) issue_qk();
+                if (ok && n >= kQkLead) issue_pv();
             }
 #endif
             PROF_END(kProfMmaTotal);
@@ -686,6 +723,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             bool ok = true;
             float l[HPT];
             int trace_n = (ws == 0) ? 0 : 100000; (void)trace_n;
+            struct { bool valid, whole; int b, seg, slot_id, c_nt; long long c_P; float m_mine; } pend;
+            pend.valid = false;
             // Only the first softmax warp watches an mbarrier; the others are released through the named
             // barrier, which also makes the outcome uniform across the group.
             auto group_wait = [&](void* bar, uint32_t parity) -> bool {
@@ -696,6 +735,69 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 if (ws == 0) failed = !mbar_wait(bar, parity, abort_flag);
                 return !softmax_bar_or(failed, NSM);
 #endif
+            };
+            // Output of a finished segment: normalised rows straight to `out`, or the unnormalised partial result.
+            auto run_epilogue = [&]() -> bool {
+                const int set = pend.seg & 1, b = pend.b;
+                const bool whole = pend.whole;
+                pend.valid = false;
+                { PROF_BEGIN();
+                  if (!group_wait(&bars.o_full[set], (pend.seg >> 1) & 1)) return false;
+                  PROF_END(kProfSmOFull); }
+                tc_fence_after();
+                TRACE(2, 41, pend.seg);
+                PROF_BEGIN();
+                float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, pend.slot_id);
+                const int Hp4 = round_up(H, 4);
+                if (!whole && sid < H) {
+                    slot_ptr[sid] = pend.m_mine;
+                    slot_ptr[Hp4 + sid] = misc.lsum[set][sid];
+                }
+                float o[NACC][HPT];
+#pragma unroll
+                for (int j = 0; j < NACC; ++j) tmem_ld16(lane_base + kOCol + (uint32_t)(set * 128 + j * 64 + hb), o[j]);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.o_empty[set]);   // the accumulators are in registers now
+                TRACE(2, 42, pend.seg);
+                if (whole) {
+                    float inv[HPT];
+#pragma unroll
+                    for (int i = 0; i < HPT; ++i) inv[i] = __frcp_rn(misc.lsum[set][hb + i]);
+#pragma unroll
+                    for (int j = 0; j < NACC; ++j) {
+                        float* dst = p.out + ((size_t)b * H + hb) * D + j * 128 + row;
+#pragma unroll
+                        for (int i = 0; i < HPT; ++i)
+                            if (hb + i < H) dst[(size_t)i * D] = o[j][i] * inv[i];
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < NACC; ++j) {
+                        float* dst = slot_ptr + 2 * Hp4 + (size_t)hb * D + j * 128 + row;
+#pragma unroll
+                        for (int i = 0; i < HPT; ++i)
+                            if (hb + i < H) dst[(size_t)i * D] = o[j][i];
+                    }
+                    // Publish this partial result.  The block that delivers a sequence's last partial result
+                    // merges all of them after its own tiles are done (merge_sequence).
+                    __threadfence();
+                    softmax_bar_sync(NSM);
+                    if (sid == 0) {
+                        const int i_first = cta_of_tile(pend.c_P, T, G), i_last = cta_of_tile(pend.c_P + pend.c_nt - 1, T, G);
+                        const int nparts = (T >= G) ? (i_last - i_first + 1) : pend.c_nt;   // T < G: one tile per block
+                        const int old = atomicAdd(ws_arrivals(p.workspace, p.B) + b, 1);
+                        if (old == nparts - 1) {
+                            __threadfence();
+                            const int k = misc.n_pending++;
+                            misc.pending[k] = b; misc.pending_p[k] = (int)pend.c_P; misc.pending_nt[k] = pend.c_nt;
+                        }
+                    }
+                }
+                TRACE(2, 43, pend.seg);
+                PROF_END(kProfSmEpilogue);
+                return true;
             };
             PROF_BEGIN();
 #ifdef MQA_X_LOADONLY
@@ -721,23 +823,26 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 softmax_bar_sync(NSM);
                 bool first = true;
                 for (;;) {
-                    const int sb = ns & 1;
+                    const int sb = ns & 3;
                     const int nvalid = c.nvalid();
                     const bool last = c.last_in_seg();
                     { PROF_BEGIN();
-                      if (!group_wait(&bars.s_full[sb], (ns >> 1) & 1)) { ok = false; break; }
+                      if (!group_wait(&bars.s_full[sb], (ns >> 2) & 1)) { ok = false; break; }
                       PROF_END(kProfSmSFull); }
                     tc_fence_after();
                     TRACE(2, 30, ns);   // S ready
                     float y[HPT];
+                    { PROF_BEGIN();
                     tmem_ld16(lane_base + (uint32_t)(sb * 64 + hb), y);
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars.s_empty[sb]);   // one arrival per warp
+                    PROF_END(kProfSmLoad); }
                     const bool valid = row < nvalid;
                     // y = scale_log2 * logit (-inf for rows beyond the sequence); does any y exceed m + threshold?
                     float xmax = -INFINITY;
+                    PROF_BEGIN();
 #pragma unroll
                     for (int i = 0; i < HPT; i += 4) {
                         const float4 mm = *reinterpret_cast<const float4*>(&misc.m[hb + i]);
@@ -748,10 +853,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         // fmaxf drops the NaN of (-inf) - (-inf)
                         xmax = fmaxf(fmaxf(xmax, fmaxf(y[i] - mm.x, y[i + 1] - mm.y)), fmaxf(y[i + 2] - mm.z, y[i + 3] - mm.w));
                     }
+                    PROF_END(kProfSmScale);
                     bool need;
                     { PROF_BEGIN(); need = softmax_bar_or(xmax > kRescaleThreshold, NSM); PROF_END(kProfSmBar); }
                     TRACE(2, 31, ns);   // after bar.red
-                    bool waited_p_empty = false;
                     if (need) {
                         // exact per-head maximum of this tile; move the reference m up and rescale l and O
                         PROF_BEGIN();
@@ -773,13 +878,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         for (int i = 0; i < HPT; ++i) l[i] *= misc.alpha[hb + i];
                         if (!first) {
                             // the accumulators can be rescaled once the MMAs of tile ns-1 have completed
-                            if (!group_wait(&bars.p_empty, (ns & 1) ^ 1)) { ok = false; break; }
-                            waited_p_empty = true;
+                            if (!group_wait(&bars.p_empty[(ns - 1) % kPBufs], ((ns - 1) / kPBufs) & 1)) { ok = false; break; }
                             tc_fence_after();
 #pragma unroll
                             for (int j = 0; j < NACC; ++j) {
                                 float o[HPT];
-                                const uint32_t ta = lane_base + 128u + (uint32_t)(j * 64 + hb);
+                                const uint32_t ta = lane_base + kOCol + (uint32_t)((seg & 1) * 128 + j * 64 + hb);
                                 tmem_ld16(ta, o);
                                 tmem_wait_ld();
 #pragma unroll
@@ -811,17 +915,18 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         PROF_END(kProfSmStore);
                     }
                     TRACE(2, 32, ns);   // p packed
-                    // the probabilities of tile ns overwrite the buffer read by the MMAs of tile ns-1
-                    if (!waited_p_empty) {
+                    // the probabilities go to one of two buffers
+                    {   // buffer ns&1 was last read by the MMAs of tile ns-2
                         PROF_BEGIN();
-                        if (!group_wait(&bars.p_empty, (ns & 1) ^ 1)) { ok = false; break; }
+                        if (!group_wait(&bars.p_empty[ns % kPBufs], ((ns / kPBufs) & 1) ^ 1)) { ok = false; break; }
                         PROF_END(kProfSmPEmpty);
                     }
                     TRACE(2, 33, ns);   // p_empty seen
                     {
+                        PROF_BEGIN();
                         // MN-major, 128B-swizzled B operand: one 128-byte row per cache row, heads contiguous
-                        unsigned char* ph = p_hi + row * 128;
-                        unsigned char* pl = p_lo + row * 128;
+                        unsigned char* ph = p_buf + (ns % kPBufs) * (2 * L::kPBytes) + row * 128;
+                        unsigned char* pl = ph + L::kPBytes;
 #pragma unroll
                         for (int u = 0; u < HPT / 8; ++u) {
                             const uint32_t unit = (uint32_t)(hb / 8 + u);
@@ -830,36 +935,26 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                             if (use_lo)
                                 *reinterpret_cast<uint4*>(pl + off) = make_uint4(lw[4 * u], lw[4 * u + 1], lw[4 * u + 2], lw[4 * u + 3]);
                         }
-                    }
-                    if (nvalid < kTileRows) {
-                        // rows beyond the sequence may hold any bits: zero them in the staged V tile
-                        const int s0 = item_of_v(ns, N) * SPT;
-                        for (int vi = 0; vi < SPT; ++vi) {
-                            const int r = vi / NACC;
-                            const int s = s0 + vi, slot = s % nslots, use = s / nslots;
-                            if (!group_wait(&bars.full[slot], use & 1)) { ok = false; break; }
-                            if (hb == 0 && !valid && (row >> 6) == r) {
-                                uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (row & 63) * 128);
-                                uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + (row & 63) * 128);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) { dst0[i] = make_uint4(0, 0, 0, 0); dst1[i] = make_uint4(0, 0, 0, 0); }
-                            }
-                        }
-                        if (!ok) break;
-                    }
                     fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars.p_full);
+                    if (lane == 0) mbar_arrive(&bars.p_full[ns % kPBufs]);
+                    PROF_END(kProfSmPublish); }
                     TRACE(2, 34, ns);   // P published
+                    if (first && pend.valid) {   // the previous segment's output, overlapped with this segment's MMAs
+                        if (!run_epilogue()) { ok = false; break; }
+                    }
                     first = false;
                     ++ns;
                     c.advance();
                     if (last) break;
                 }
                 if (!ok) break;
-                // ---------------- segment epilogue ----------------
-                const float m_mine = (sid < HP) ? misc.m[sid] : 0.f;
-                // row sums over the 128 cache-row lanes
+                // ---------------- segment end: row sums now, output later ----------------
+                // The accumulators of this segment are final only when its last MMAs complete.  Instead of draining
+                // the pipeline here, the output is written after the first tile of the NEXT segment has been handed
+                // to the MMA issuer (the two segments use different accumulator sets in tensor memory).
+                TRACE(2, 40, ns);
+                pend.m_mine = (sid < HP) ? misc.m[sid] : 0.f;
 #pragma unroll
                 for (int i = 0; i < HPT; ++i) {
                     float v = l[i];
@@ -868,62 +963,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     if (lane == i) misc.wred[wq][hb + i] = v;
                 }
                 softmax_bar_sync(NSM);
-                if (sid < HP) misc.alpha[sid] = (misc.wred[0][sid] + misc.wred[1][sid]) + (misc.wred[2][sid] + misc.wred[3][sid]);
-                softmax_bar_sync(NSM);     // misc.alpha now holds the row sums l[h]
-                { PROF_BEGIN();
-                  if (!group_wait(&bars.o_full, seg & 1)) { ok = false; break; }
-                  PROF_END(kProfSmOFull); }
-                tc_fence_after();
-                {
-                PROF_BEGIN();
-                float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, slot_id);
-                const int Hp4 = round_up(H, 4);
-                if (!whole && sid < H) {
-                    slot_ptr[sid] = m_mine;
-                    slot_ptr[Hp4 + sid] = misc.alpha[sid];
-                }
-                float o[NACC][HPT];
-#pragma unroll
-                for (int j = 0; j < NACC; ++j) tmem_ld16(lane_base + 128u + (uint32_t)(j * 64 + hb), o[j]);
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.o_empty);   // the accumulators are in registers: the next segment may overwrite them
-#pragma unroll
-                for (int j = 0; j < NACC; ++j) {
-                    const int d = j * 128 + row;
-                    if (whole) {
-                        float* dst = p.out + ((size_t)b * H + hb) * D + d;
-#pragma unroll
-                        for (int i = 0; i < HPT; ++i)
-                            if (hb + i < H) dst[(size_t)i * D] = o[j][i] * __frcp_rn(misc.alpha[hb + i]);
-                    } else {
-                        float* dst = slot_ptr + 2 * Hp4 + (size_t)hb * D + d;
-#pragma unroll
-                        for (int i = 0; i < HPT; ++i)
-                            if (hb + i < H) dst[(size_t)i * D] = o[j][i];
-                    }
-                }
-                if (!whole) {
-                    // Publish this partial result.  The block that delivers a sequence's last partial result
-                    // merges all of them after its own tiles are done (merge_sequence below).
-                    __threadfence();
-                    softmax_bar_sync(NSM);
-                    if (sid == 0) {
-                        const int i_first = cta_of_tile(c_P, T, G), i_last = cta_of_tile(c_P + c_nt - 1, T, G);
-                        const int nparts = (T >= G) ? (i_last - i_first + 1) : c_nt;   // T < G: one tile per block
-                        const int old = atomicAdd(ws_arrivals(p.workspace, p.B) + b, 1);
-                        if (old == nparts - 1) {
-                            __threadfence();
-                            const int k = misc.n_pending++;
-                            misc.pending[k] = b; misc.pending_p[k] = (int)c_P; misc.pending_nt[k] = c_nt;
-                        }
-                    }
-                }
-                softmax_bar_sync(NSM);     // misc.m / misc.alpha are rewritten by the next segment
-                PROF_END(kProfSmEpilogue);
-                }
+                if (sid < HP) misc.lsum[seg & 1][sid] = (misc.wred[0][sid] + misc.wred[1][sid]) + (misc.wred[2][sid] + misc.wred[3][sid]);
+                softmax_bar_sync(NSM);
+                pend.valid = true; pend.b = b; pend.seg = seg; pend.whole = whole; pend.slot_id = slot_id;
+                pend.c_P = c_P; pend.c_nt = c_nt;
             }
+            if (ok && pend.valid) ok = run_epilogue();
             PROF_END(kProfSmTotal);
         }
     }
