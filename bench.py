@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the multiquery decode-attention hot path on B200.
 
-One step = one whole pass of the path (split kernel + combine kernel) over one
-batch of synthetic PaLM-shaped input.  Prints ONE JSON line (rank 0).
+One step = one whole pass of the path (the split kernel, which also merges the
+sequences it cuts; on the FMA path a separate combine kernel) over one batch of
+synthetic PaLM-shaped input.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
@@ -45,6 +46,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_traffic(workload_name):
+    """DRAM bytes per launch of the split kernel from the committed ncu summary, if there is one."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f).get(workload_name)
+    except Exception:
+        return None
+
+
 def config_of(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: B={w.B} H={w.H} D={w.D} Lmax={w.Lmax} "
                        f"{'ragged lengths' if w.ragged else 'uniform lengths'} bf16 q/K/V fp32 out",
@@ -71,7 +81,7 @@ class ClockSampler:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -188,6 +198,11 @@ def run_ours(args, w):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        # nvidia-smi needs a moment to start sampling; keep the GPU under the same load meanwhile
+        t_spin = time.perf_counter()
+        while time.perf_counter() - t_spin < args.clock_spin_s:
+            step()
+        torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
            torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for a, m, b in ev:          # force creation of the event handles
@@ -282,7 +297,7 @@ def run_ours(args, w):
         "pct_of_measured_copy_peak": 100.0 * value / world / peak,
         "roofline": {"bound": "hbm", "kernel": "split kernel (mqa_fma/mqa_tc)", "achieved": achieved, "peak": peak,
                      "peak_kind": f"{peak_kind} STREAM-style copy", "unit": "GB/s", "frac": achieved / peak,
-                     "kernel_us": main_ms_avg * 1e3, "traffic": None},
+                     "kernel_us": main_ms_avg * 1e3, "traffic": measured_traffic(w.name)},
         "cpu_baseline": cpu,
         "e2e": e2e,
         "gpu_launches": launches_per_step * args.steps,
@@ -303,6 +318,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--clock-spin-s", type=float, default=0.3,
+                    help="seconds of extra untimed load while the clock sampler starts (0 under a profiler)")
     ap.add_argument("--ref-sample-seqs", type=int, default=512,
                     help="sequences of the workload the CPU oracle is timed on")
     args = ap.parse_args()

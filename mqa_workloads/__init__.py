@@ -44,6 +44,8 @@ WORKLOADS = {
     "palm8b": Workload("palm8b", B=8, H=16, D=256, Lmax=2048, seed=221105102),
     "palm62b": Workload("palm62b", B=64, H=32, D=256, Lmax=2048, seed=221105103),
     "palm540b": Workload("palm540b", B=512, H=48, D=256, Lmax=2048, seed=221105104),
+    # one eighth of palm540b (same H, D, L): small enough for multi-pass profiler captures
+    "palm540b_b64": Workload("palm540b_b64", B=64, H=48, D=256, Lmax=2048, seed=221105106),
     "ragged32k": Workload("ragged32k", B=16, H=48, D=256, Lmax=32768, seed=221105105,
                           ragged=True, k_outlier_frac=0.01, k_outlier_var=2.0),
 }
