@@ -67,7 +67,7 @@ def config_of(w, n_gpus, extra=None):
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -86,8 +86,11 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and active throttle reasons over the samples taken in [t_begin, t_end]
+        (time.time() values; all samples if the window holds none)."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         time.sleep(0.15)
@@ -98,23 +101,27 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.file:
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]),
+                             [nm for nm, val in zip(names, f[4:8]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, f[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
         self.file.close()
         os.unlink(self.file.name)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if t_begin is not None and t_begin - 0.01 <= r[0] <= t_end + 0.01]
+        use = inside or rows
+        if use:
+            reasons = sorted({nm for r in use for nm in r[4]})
+            out.update(sm_mhz=statistics.median(r[1] for r in use), sm_max_mhz=max(r[2] for r in use),
+                       power_w=statistics.median(r[3] for r in use), reasons=reasons, samples=len(use),
+                       window="timed region" if inside else "whole run (no sample fell inside the timed region)")
         return out
 
 
@@ -188,6 +195,10 @@ def run_ours(args, w):
             flush.fill_(1)
         binding.mqa_decode(qd, kd, vd, ld, out, w.scale, ws, stream=stream, plan=plan)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0 and args.clock_spin_s > 0:
+        sampler.start()
+        time.sleep(args.clock_spin_s)      # nvidia-smi needs a moment before its first sample
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -195,14 +206,6 @@ def run_ours(args, w):
     launches_per_step = binding.mqa_last_launch_count()
 
     # ---- timed region: K steps, each bracketed by events so flush time is excluded ----
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        # nvidia-smi needs a moment to start sampling; keep the GPU under the same load meanwhile
-        t_spin = time.perf_counter()
-        while time.perf_counter() - t_spin < args.clock_spin_s:
-            step()
-        torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
            torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for a, m, b in ev:          # force creation of the event handles
@@ -210,6 +213,7 @@ def run_ours(args, w):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
+    t_begin = time.time()
     wall0 = time.perf_counter()
     for a, m, b in ev:
         if flush is not None:
@@ -221,7 +225,7 @@ def run_ours(args, w):
     if dist is not None:
         dist.barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, time.time()) if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, m, b in ev]
     main_ms = [a.elapsed_time(m) for a, m, b in ev]          # split kernel only
     total_ms = sum(step_ms)
@@ -314,12 +318,12 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--clock-spin-s", type=float, default=0.3,
-                    help="seconds of extra untimed load while the clock sampler starts (0 under a profiler)")
+                    help="seconds to let the nvidia-smi clock sampler start before the warm-up (0 = no sampling)")
     ap.add_argument("--ref-sample-seqs", type=int, default=512,
                     help="sequences of the workload the CPU oracle is timed on")
     args = ap.parse_args()
