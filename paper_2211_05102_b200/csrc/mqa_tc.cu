@@ -30,7 +30,7 @@ namespace {
 constexpr int kHeadsPerThread = 16;        // a softmax thread owns one cache row and 16 heads
 constexpr int kTileShift = 7;
 constexpr int kTileRows = 128;
-constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 64 rows x 128 cols (V)
+constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 8192/D whole rows (V)
 constexpr int kMaxSlots = 12;
 constexpr int kMinSlots = 4;               // any depth >= 1 is deadlock-free (slots are filled and drained in one order)
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logit units: rescale only when a logit exceeds m + 8
@@ -380,6 +380,7 @@ struct TcLayout {
     static constexpr int kThreads = 128 + kSoftmaxThreads;   // warps 0-3: producer, MMA issuer, two idle
     static constexpr int SPT = D / 64;            // ring slots per K tile and per V tile
     static constexpr int NACC = D / 128;          // 128-wide halves of D = output accumulators
+    static constexpr int VROWS = 8192 / D;        // cache rows per V slot: a slot is VROWS full rows, contiguous in global memory
     static constexpr int kQBytes = HP * D * 2;    // one q buffer: D/64 chunks of [HP rows x 128 B]
     static constexpr int kPBytes = 128 * 128;     // one probability buffer: 128 cache rows x 128 B (up to 64 heads)
     static constexpr int kFixed = 2 * kQBytes + 2 * kPBufs * kPBytes + (int)sizeof(Misc);   // q x2, (hi, lo) x kPBufs
@@ -513,7 +514,6 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             auto load_v = [&](const TileCursor& c) {
 #pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
-                    const int r = vi / NACC, j = vi % NACC;
                     const int slot = pslot;
 #ifndef MQA_X_NOCHUNKSYNC
                     {
@@ -531,8 +531,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         (void)dst; mbar_arrive(&bars.full[slot]);
 #else
                         mbar_expect_tx(&bars.full[slot], kSlotBytes);
-                        tma_load_3d(dst, &map_v, &bars.full[slot], j * 128, c.row0() + r * 64, c.w.b, policy);
-                        tma_load_3d(dst + 8192, &map_v, &bars.full[slot], j * 128 + 64, c.row0() + r * 64, c.w.b, policy);
+                        // D/64 boxes of [VROWS rows x 64 columns]: together VROWS whole rows, 16 KB contiguous in global memory
+#pragma unroll
+                        for (int cb = 0; cb < D / 64; ++cb)
+                            tma_load_3d(dst + cb * (L::VROWS * 128), &map_v, &bars.full[slot], cb * 64, c.row0() + vi * L::VROWS, c.w.b, policy);
 #endif
                     }
                     __syncwarp();
@@ -570,7 +572,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             int trace_n = 0; (void)trace_n;
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(q_buf));
             const uint32_t ring_lo_k = desc_lo_kmajor(smem_u32(ring));
-            const uint32_t ring_lo_mn = desc_lo_mnmajor(smem_u32(ring), 8192);
+            const uint32_t ring_lo_mn = desc_lo_mnmajor(smem_u32(ring), L::VROWS * 128);
             const uint32_t p_lo32 = desc_lo_mnmajor(smem_u32(p_buf), 8192);
             PROF_BEGIN();
             auto issue_qk = [&]() {
@@ -642,7 +644,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 #pragma unroll
                 for (int vi = 0; vi < SPT; ++vi) {
                     constexpr int kStep = 2048 >> 4;               // 16 cache rows of 128 B
-                    const int r = vi / NACC, j = vi % NACC;
+                    constexpr int VR = L::VROWS;                   // rows of this slot: [vi*VR, vi*VR + VR)
                     const int slot = cslot;
 #ifndef MQA_X_NOCHUNKSYNC
                     { PROF_BEGIN();
@@ -650,37 +652,40 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                       PROF_END(kProfMmaVFull); }
 #endif
                     if (++cslot == nslots) { cslot = 0; cphase ^= 1; }
-                    if (nvalid < kTileRows) {
+                    if (nvalid < (vi + 1) * VR) {
                         // Rows beyond the sequence may hold any bits (0 * NaN would poison the accumulator): zero them
                         // in the staged tile.  This warp consumes the ring strictly in order, so the slot is known to
                         // hold this tile.
-                        for (int lr = max(0, nvalid - r * 64) + lane; lr < 64; lr += 32) {
-                            uint4* dst0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + lr * 128);
-                            uint4* dst1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + 8192 + lr * 128);
+                        for (int lr = max(0, nvalid - vi * VR) + lane; lr < VR; lr += 32) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) { dst0[i] = make_uint4(0, 0, 0, 0); dst1[i] = make_uint4(0, 0, 0, 0); }
+                            for (int cb = 0; cb < D / 64; ++cb) {
+                                uint4* dst = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + cb * (VR * 128) + lr * 128);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0, 0, 0, 0);
+                            }
                         }
                         fence_proxy_async();
                         __syncwarp();
                     }
                     tc_fence_after();
                     TRACE(1, 21 + vi, np);   // V slot landed
-                    const uint32_t d_tmem = tmem + kOCol + (uint32_t)((iv.seg & 1) * 128 + j * 64);
+                    const uint32_t d_tmem0 = tmem + kOCol + (uint32_t)((iv.seg & 1) * 128);
                     const uint32_t alo = ring_lo_mn + (uint32_t)slot * (kSlotBytes >> 4);
-                    const uint32_t bhl = p_lo32 + (uint32_t)(((np % kPBufs) * 2 * L::kPBytes + r * 64 * 128) >> 4);
+                    const uint32_t bhl = p_lo32 + (uint32_t)(((np % kPBufs) * 2 * L::kPBytes + vi * VR * 128) >> 4);
                     const uint32_t bll = bhl + (uint32_t)(L::kPBytes >> 4);
                     if (elect_one_sync()) {
 #ifndef MQA_X_SKIP_PV
-                        // the first MMA of a segment's accumulator overwrites it
-                        if (r == 0 && fresh) umma_bf16_lo<false>(d_tmem, alo, bhl, kDescHiSw128, idesc_pv);
-                        else                 umma_bf16_lo<true>(d_tmem, alo, bhl, kDescHiSw128, idesc_pv);
 #pragma unroll
-                        for (int ks = 1; ks < 4; ++ks)             // 4 x 16 cache rows per 64-row slot
-                            umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * kStep), bhl + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
-                        if (use_lo) {
+                        for (int ks = 0; ks < VR / 16; ++ks) {     // 16 cache rows per MMA
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                umma_bf16_lo<true>(d_tmem, alo + (uint32_t)(ks * kStep), bll + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
+                            for (int j = 0; j < NACC; ++j) {       // the two 128-column halves of D
+                                const uint32_t a = alo + (uint32_t)(((2 * j) * (VR * 128)) >> 4) + (uint32_t)(ks * kStep);
+                                const uint32_t d_tmem = d_tmem0 + (uint32_t)(j * 64);
+                                // the first MMA into a segment's accumulator overwrites it
+                                if (vi == 0 && ks == 0 && fresh) umma_bf16_lo<false>(d_tmem, a, bhl + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
+                                else                             umma_bf16_lo<true>(d_tmem, a, bhl + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
+                                if (use_lo) umma_bf16_lo<true>(d_tmem, a, bll + (uint32_t)(ks * kStep), kDescHiSw128, idesc_pv);
+                            }
                         }
 #endif
 #ifndef MQA_X_NOCHUNKSYNC
@@ -776,7 +781,11 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         float* dst = p.out + ((size_t)b * H + hb) * D + j * 128 + row;
 #pragma unroll
                         for (int i = 0; i < HPT; ++i)
+#ifdef MQA_X_NOSTORE
+                            if (hb + i < H && inv[i] == 12345.f) dst[(size_t)i * D] = o[j][i] * inv[i];
+#else
                             if (hb + i < H) dst[(size_t)i * D] = o[j][i] * inv[i];
+#endif
                     }
                 } else {
 #pragma unroll
@@ -1087,7 +1096,7 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
     thread_local MapCache mc;
     if (mc.q != p.q || mc.k != p.k || mc.v != p.v || mc.B != p.B || mc.H != p.H || mc.D != p.D || mc.Lmax != p.Lmax || mc.hp != HP) {
         if (!encode_map(&mc.mq, p.q, p.D, p.H, p.B, HP) || !encode_map(&mc.mk, p.k, p.D, p.Lmax, p.B, 128) ||
-            !encode_map(&mc.mv, p.v, p.D, p.Lmax, p.B, 64)) {
+            !encode_map(&mc.mv, p.v, p.D, p.Lmax, p.B, L::VROWS)) {
             mc.q = nullptr;
             return cudaErrorInvalidValue;
         }
