@@ -56,7 +56,8 @@ typedef enum {
     MQA_ERR_WORKSPACE_TOO_SMALL = 4,
     MQA_ERR_ARCH = 5,                /* current device is not compute capability 10.x      */
     MQA_ERR_CUDA = 6,                /* a CUDA runtime/driver call failed                  */
-    MQA_ERR_TIMEOUT = 7              /* a bounded device-side wait ran out (see check_status) */
+    MQA_ERR_TIMEOUT = 7,             /* a bounded device-side wait ran out (see check_status) */
+    MQA_ERR_CACHE_FULL = 8           /* mqa_append_decode: some sequence had no free cache row (see check_status) */
 } mqa_status_t;
 
 /* Kernel families (mqa_plan_t.path). */
@@ -129,7 +130,25 @@ int mqa_decode(const void* q, const void* k_cache, const void* v_cache,
                int B, int H, int D, int Lmax, float scale,
                void* workspace, size_t workspace_bytes, void* stream);
 
-/* Same, with an explicit plan (tests and tuning). */
+/*
+ * One whole generate step of the attention layer (Section 2.2: every decode step yields one new token
+ * per sequence whose key/value joins the cache; Section 3.3: that step has one token of Q, K, V per
+ * sequence against a cache of many): append, then attend.
+ *   k_new, v_new  device bf16 [B,D]   this step's key and value row of every sequence, 16-byte aligned
+ *   k_cache, v_cache                  device bf16 [B,Lmax,D], WRITTEN: row lengths[b] of sequence b
+ *   lengths       device int32 [B]    in: valid rows before the step; out: incremented by one
+ * For every b with 0 <= lengths[b] < Lmax the new rows are stored at index lengths[b] and lengths[b]
+ * grows by one; then out is computed exactly as by mqa_decode over the lengthened cache.  A sequence
+ * with lengths[b] >= Lmax (or negative) gets nothing appended, keeps its length, is attended over its
+ * clamped old length, and MQA_ERR_CACHE_FULL is recorded in the workspace status word (read it with
+ * mqa_check_status).  Two kernels are enqueued (append, split); other arguments as in mqa_decode.
+ */
+int mqa_append_decode(const void* q, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, int32_t* lengths, float* out,
+                      int B, int H, int D, int Lmax, float scale,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same as mqa_decode, with an explicit plan (tests and tuning). */
 int mqa_decode_with_plan(const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* lengths, float* out,
                          int B, int H, int D, int Lmax, float scale,
@@ -151,8 +170,9 @@ int mqa_decode_profiled(const void* q, const void* k_cache, const void* v_cache,
 
 /*
  * Synchronise `stream`, read the device status word from the workspace header,
- * reset it to zero and return it (MQA_OK, or MQA_ERR_TIMEOUT if a bounded wait
- * inside a kernel gave up; the output of that call is then undefined).
+ * reset it to zero and return it (MQA_OK; MQA_ERR_TIMEOUT if a bounded wait
+ * inside a kernel gave up, the output of that call is then undefined;
+ * MQA_ERR_CACHE_FULL after mqa_append_decode found a full cache).
  */
 int mqa_check_status(void* workspace, void* stream);
 

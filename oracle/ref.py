@@ -152,3 +152,26 @@ def mqa_ref_merge(m: np.ndarray, z: np.ndarray, acc: np.ndarray) -> np.ndarray:
     if rc != 0:
         raise RuntimeError("mqa_ref_merge_f64 failed")
     return out
+
+
+def mqa_append_decode_ref(q, k_new, v_new, k, v, lengths, scale: float, num_threads: int | None = None):
+    """One generate step of the attention layer: the step's new key/value row of every sequence joins
+    its cache (paper Section 2.2: each decode step produces one token per sequence; Section 3.3: that
+    step has one token of Q, K and V per sequence against a cache of many), then the query attends over
+    the lengthened cache by the plain definition.
+
+    Returns (out[B,H,D] float64, k_bits, v_bits, new_lengths) with the caches as uint16 bf16 bit arrays.
+    A sequence whose length is outside [0, Lmax) gets nothing appended and keeps its length.
+    """
+    qb, kb, vb, ln = as_bits(q), as_bits(k).copy(), as_bits(v).copy(), _lens(lengths).copy()
+    knb, vnb = as_bits(k_new), as_bits(v_new)
+    B, Lmax, D = kb.shape
+    assert knb.shape == (B, D) and vnb.shape == (B, D)
+    for b in range(B):
+        n = int(ln[b])
+        if 0 <= n < Lmax:
+            kb[b, n, :] = knb[b]
+            vb[b, n, :] = vnb[b]
+            ln[b] = n + 1
+    out = mqa_decode_ref(qb, kb, vb, ln, scale, num_threads)
+    return out, kb, vb, ln

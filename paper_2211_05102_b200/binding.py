@@ -22,6 +22,7 @@ MQA_ERR_WORKSPACE_TOO_SMALL = 4
 MQA_ERR_ARCH = 5
 MQA_ERR_CUDA = 6
 MQA_ERR_TIMEOUT = 7
+MQA_ERR_CACHE_FULL = 8
 
 MQA_PATH_AUTO = 0
 MQA_PATH_FMA = 1
@@ -31,7 +32,7 @@ MQA_MAX_CTAS = 592
 EXPORTS = [
     "mqa_status_string", "mqa_decode_workspace_bytes", "mqa_workspace_init", "mqa_decode_plan",
     "mqa_decode", "mqa_decode_with_plan", "mqa_decode_profiled", "mqa_check_status", "mqa_decode_host_scratch_bytes",
-    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static",
+    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static", "mqa_append_decode",
 ]
 
 
@@ -74,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_host.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, sz, vp]; L.mqa_decode_host.restype = ci
         L.mqa_last_launch_count.argtypes = []; L.mqa_last_launch_count.restype = ci
         L.mqa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp]; L.mqa_decode_static.restype = ci
+        L.mqa_append_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, sz, vp]
+        L.mqa_append_decode.restype = ci
         L.mqa_debug_schedule.argtypes = [vp, ci, ci, ci, ci, ci, vp, ci]; L.mqa_debug_schedule.restype = ci
         _lib = L
     return _lib
@@ -181,6 +184,20 @@ def mqa_decode_static(q, k_cache, v_cache, lengths, out, scale: float, stream=No
     rc = lib().mqa_decode_static(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), lengths.data_ptr(),
                                  out.data_ptr(), B, H, D, Lmax, float(scale), _stream_ptr(stream))
     _check(rc, "mqa_decode_static")
+    return out
+
+
+def mqa_append_decode(q, k_new, v_new, k_cache, v_cache, lengths, out, scale: float, workspace, stream=None):
+    """Append this step's K/V rows to the caches (in place, lengths incremented), then attend."""
+    B, H, D, Lmax = _shapes(q, k_cache, v_cache, lengths, out)
+    assert k_new.shape == (B, D) and v_new.shape == (B, D)
+    assert k_new.dtype == torch.bfloat16 and v_new.dtype == torch.bfloat16
+    for t in (q, k_new, v_new, k_cache, v_cache, lengths, out, workspace):
+        assert t.is_cuda and t.is_contiguous()
+    rc = lib().mqa_append_decode(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), k_cache.data_ptr(),
+                                 v_cache.data_ptr(), lengths.data_ptr(), out.data_ptr(), B, H, D, Lmax,
+                                 float(scale), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "mqa_append_decode")
     return out
 
 

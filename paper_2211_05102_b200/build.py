@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmqa_decode.so")
-SOURCES = ["mqa_api.cu", "mqa_fma.cu", "mqa_combine.cu", "mqa_tc.cu", "mqa_static_ws.cu"]
+SOURCES = ["mqa_api.cu", "mqa_fma.cu", "mqa_combine.cu", "mqa_tc.cu", "mqa_static_ws.cu", "mqa_append.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 

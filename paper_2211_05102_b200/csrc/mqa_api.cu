@@ -48,6 +48,7 @@ const char* mqa_status_string(int status)
         case MQA_ERR_ARCH: return "device is not compute capability 10.x";
         case MQA_ERR_CUDA: return "CUDA call failed";
         case MQA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case MQA_ERR_CACHE_FULL: return "a sequence's cache had no free row for the appended token";
         default: return "unknown status";
     }
 }
@@ -183,6 +184,38 @@ int mqa_decode(const void* q, const void* k_cache, const void* v_cache,
     if (rc != MQA_OK) return rc;
     return mqa_decode_with_plan(q, k_cache, v_cache, lengths, out, B, H, D, Lmax, scale, &plan,
                                 workspace, workspace_bytes, stream);
+}
+
+int mqa_append_decode(const void* q, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, int32_t* lengths, float* out,
+                      int B, int H, int D, int Lmax, float scale,
+                      void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!q || !k_new || !v_new || !k_cache || !v_cache || !lengths || !out || !workspace) return MQA_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || D <= 0 || Lmax <= 0) return MQA_ERR_INVALID_ARG;
+    if (!shape_ok(B, H, D, Lmax)) return MQA_ERR_UNSUPPORTED_SHAPE;
+    if (!(scale == scale)) return MQA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) ||
+        !aligned(out, 16) || !aligned(lengths, 4) || !aligned(workspace, 256))
+        return MQA_ERR_MISALIGNED;
+    if (workspace_bytes < mqa::workspace_bytes(B, H, D)) return MQA_ERR_WORKSPACE_TOO_SMALL;
+    mqa_plan_t plan;
+    int rc = mqa_decode_plan(B, H, D, Lmax, MQA_PATH_AUTO, &plan);
+    if (rc != MQA_OK) return rc;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return MQA_ERR_CUDA;
+    }
+    if (major != 10) return MQA_ERR_ARCH;
+    if (mqa::launch_append(k_new, v_new, k_cache, v_cache, lengths, B, D, Lmax,
+                           static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return MQA_ERR_CUDA;
+    rc = decode_impl(q, k_cache, v_cache, lengths, out, B, H, D, Lmax, scale, &plan, workspace, workspace_bytes,
+                     stream, nullptr);
+    if (rc == MQA_OK) g_last_launches += 1;
+    return rc;
 }
 
 int mqa_check_status(void* workspace, void* stream)

@@ -187,6 +187,8 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 cudaError_t launch_fma(const Params& p, cudaStream_t stream);
 cudaError_t launch_combine(const Params& p, cudaStream_t stream);
 cudaError_t launch_tc(const Params& p, cudaStream_t stream);
+cudaError_t launch_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int32_t* lengths,
+                          int B, int D, int Lmax, unsigned char* workspace, cudaStream_t stream);
 bool tc_supported(int H, int D);
 
 }  // namespace mqa

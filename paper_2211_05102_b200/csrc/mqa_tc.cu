@@ -784,7 +784,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 #ifdef MQA_X_NOSTORE
                             if (hb + i < H && inv[i] == 12345.f) dst[(size_t)i * D] = o[j][i] * inv[i];
 #else
-                            if (hb + i < H) dst[(size_t)i * D] = o[j][i] * inv[i];
+                            if (hb + i < H) __stcs(dst + (size_t)i * D, o[j][i] * inv[i]);
 #endif
                     }
                 } else {

@@ -33,8 +33,8 @@ def test_header_symbols_are_exported(L):
 
 
 def test_status_strings(L):
-    seen = {binding.status_string(i) for i in range(8)}
-    assert len(seen) == 8
+    seen = {binding.status_string(i) for i in range(9)}
+    assert len(seen) == 9
     assert binding.status_string(1234) == "unknown status"
 
 
@@ -95,6 +95,12 @@ def test_argument_errors_launch_nothing(L):
     assert _call(L, plan=binding.Plan(binding.MQA_PATH_FMA, 4, 128)) == binding.MQA_ERR_INVALID_ARG
     assert _call(L, plan=binding.Plan(7, 4, 64)) == binding.MQA_ERR_INVALID_ARG
     assert _call(L, plan=binding.Plan(binding.MQA_PATH_TC, 4, 128)) == binding.MQA_ERR_UNSUPPORTED_SHAPE  # D=64
+    assert L.mqa_append_decode(0x1000, None, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 2, 4, 64, 128, 0.1, 0x10000, 1 << 26, None) \
+        == binding.MQA_ERR_INVALID_ARG
+    assert L.mqa_append_decode(0x1000, 0x2008, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 2, 4, 64, 128, 0.1, 0x10000, 1 << 26, None) \
+        == binding.MQA_ERR_MISALIGNED
+    assert L.mqa_append_decode(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 2, 4, 64, 128, 0.1, 0x10000, 512, None) \
+        == binding.MQA_ERR_WORKSPACE_TOO_SMALL
     assert L.mqa_check_status(None, None) == binding.MQA_ERR_INVALID_ARG
     assert L.mqa_workspace_init(None, 1 << 20, None) == binding.MQA_ERR_INVALID_ARG
     assert L.mqa_workspace_init(0x10000, 8, None) == binding.MQA_ERR_WORKSPACE_TOO_SMALL
