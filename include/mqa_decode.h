@@ -64,7 +64,7 @@ typedef enum {
 enum {
     MQA_PATH_AUTO = 0,
     MQA_PATH_FMA = 1,   /* fp32 FMA kernel, any supported shape                      */
-    MQA_PATH_TC = 2     /* tcgen05 tensor-core kernel with TMA staging: D in {128,256}, H >= 8 */
+    MQA_PATH_TC = 2     /* tcgen05 tensor-core kernel with TMA staging: D in {128,256}          */
 };
 
 /*
@@ -147,6 +147,25 @@ int mqa_append_decode(const void* q, const void* k_new, const void* v_new,
                       void* k_cache, void* v_cache, int32_t* lengths, float* out,
                       int B, int H, int D, int Lmax, float scale,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Decode attention with KVH key/value heads per sequence (grouped-query attention; KVH == H is the
+ * multihead attention the paper compares against in Section 4.2 and Table 1, KVH == 1 is mqa_decode).
+ * Query head h uses key/value head h / (H/KVH).  The cache then holds KVH times the bytes, which is the
+ * memory-time cost Section 3.3 attributes to multihead attention.
+ *   q        device bf16 [B,H,D]            the H/KVH heads of one group adjacent
+ *   k_cache  device bf16 [B,KVH,Lmax,D]     (one contiguous [Lmax,D] cache per key/value head)
+ *   v_cache  device bf16 [B,KVH,Lmax,D]
+ *   lengths  device int32 [B]               shared by the KVH heads of a sequence
+ *   out      device fp32 [B,H,D]
+ *   workspace  >= mqa_decode_grouped_workspace_bytes(B, H, KVH, D, Lmax), 256-byte aligned, initialised
+ * H must be a multiple of KVH; H/KVH and D obey the limits of mqa_decode.  Everything else as mqa_decode.
+ */
+int mqa_decode_grouped(const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* lengths, float* out,
+                       int B, int H, int KVH, int D, int Lmax, float scale,
+                       void* workspace, size_t workspace_bytes, void* stream);
+size_t mqa_decode_grouped_workspace_bytes(int B, int H, int KVH, int D, int Lmax);
 
 /* Same as mqa_decode, with an explicit plan (tests and tuning). */
 int mqa_decode_with_plan(const void* q, const void* k_cache, const void* v_cache,

@@ -228,6 +228,49 @@ int mqa_ref_merge_f64(const double* m, const double* z, const double* acc,
     return 0;
 }
 
+/*
+ * Attention with KVH key/value heads per sequence (Section 4.2 compares multihead attention, KVH = H,
+ * with multiquery attention, KVH = 1).  Query head h reads key/value head g = h / (H/KVH).
+ * Layouts: q [B,H,D], k and v [B,KVH,Lmax,D], lengths [B], out [B,H,D].  The plain definition again,
+ * written with its own index arithmetic (it does not call the multiquery routine above).
+ */
+int gqa_decode_ref_f64(const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                       const int32_t* lengths, double* out,
+                       int B, int H, int KVH, int D, int Lmax, float scale)
+{
+    if (!q || !k || !v || !lengths || !out || bad_shape(B, H, D, Lmax) || KVH <= 0 || H % KVH != 0) return -1;
+    const double sc = (double)scale;
+    const int per = H / KVH;
+    double* s = (double*)malloc(sizeof(double) * (size_t)Lmax);
+    if (!s) return -1;
+    for (int b = 0; b < B; ++b) {
+        const int n = clamp_len(lengths[b], Lmax);
+        for (int h = 0; h < H; ++h) {
+            const int g = h / per;
+            const uint16_t* qv = q + ((size_t)b * H + h) * D;
+            const uint16_t* kh = k + (((size_t)b * KVH + g) * Lmax) * D;
+            const uint16_t* vh = v + (((size_t)b * KVH + g) * Lmax) * D;
+            double* o = out + ((size_t)b * H + h) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (n == 0) continue;
+            double m = -INFINITY;
+            for (int l = 0; l < n; ++l) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += bf16_bits_to_double(qv[d]) * bf16_bits_to_double(kh[(size_t)l * D + d]);
+                s[l] = sc * acc;
+                if (s[l] > m) m = s[l];
+            }
+            double Z = 0.0;
+            for (int l = 0; l < n; ++l) { s[l] = exp(s[l] - m); Z += s[l]; }
+            for (int l = 0; l < n; ++l)
+                for (int d = 0; d < D; ++d) o[d] += s[l] * bf16_bits_to_double(vh[(size_t)l * D + d]);
+            for (int d = 0; d < D; ++d) o[d] /= Z;
+        }
+    }
+    free(s);
+    return 0;
+}
+
 int mqa_ref_max_threads(void)
 {
 #ifdef _OPENMP

@@ -54,6 +54,8 @@ def _load():
         lib.mqa_ref_partial_f64.restype = ci
         lib.mqa_ref_merge_f64.argtypes = [f64p, f64p, f64p, ci, ci, f64p]
         lib.mqa_ref_merge_f64.restype = ci
+        lib.gqa_decode_ref_f64.argtypes = [u16p, u16p, u16p, i32p, f64p, ci, ci, ci, ci, ci, ctypes.c_float]
+        lib.gqa_decode_ref_f64.restype = ci
         lib.mqa_ref_max_threads.argtypes = []
         lib.mqa_ref_max_threads.restype = ci
         _lib = lib
@@ -175,3 +177,20 @@ def mqa_append_decode_ref(q, k_new, v_new, k, v, lengths, scale: float, num_thre
             ln[b] = n + 1
     out = mqa_decode_ref(qb, kb, vb, ln, scale, num_threads)
     return out, kb, vb, ln
+
+
+def gqa_decode_ref(q, k, v, lengths, scale: float) -> np.ndarray:
+    """Reference for KVH key/value heads per sequence (Section 4.2's multihead / multiquery comparison):
+    q [B,H,D], k/v [B,KVH,Lmax,D]; query head h reads key/value head h // (H // KVH). Returns [B,H,D] float64."""
+    lib = _load()
+    qb, kb, vb, ln = as_bits(q), as_bits(k), as_bits(v), _lens(lengths)
+    B, H, D = qb.shape
+    KVH, Lmax = kb.shape[1], kb.shape[2]
+    assert kb.shape == (B, KVH, Lmax, D) and vb.shape == kb.shape and ln.shape == (B,)
+    out = np.empty((B, H, D), dtype=np.float64)
+    rc = lib.gqa_decode_ref_f64(_p(qb, ctypes.c_uint16), _p(kb, ctypes.c_uint16), _p(vb, ctypes.c_uint16),
+                                _p(ln, ctypes.c_int32), _p(out, ctypes.c_double), B, H, KVH, D, Lmax,
+                                ctypes.c_float(scale))
+    if rc != 0:
+        raise RuntimeError("gqa_decode_ref_f64 failed")
+    return out

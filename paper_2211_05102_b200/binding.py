@@ -32,7 +32,7 @@ MQA_MAX_CTAS = 592
 EXPORTS = [
     "mqa_status_string", "mqa_decode_workspace_bytes", "mqa_workspace_init", "mqa_decode_plan",
     "mqa_decode", "mqa_decode_with_plan", "mqa_decode_profiled", "mqa_check_status", "mqa_decode_host_scratch_bytes",
-    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static", "mqa_append_decode",
+    "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static", "mqa_append_decode", "mqa_decode_grouped", "mqa_decode_grouped_workspace_bytes",
 ]
 
 
@@ -77,6 +77,10 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp]; L.mqa_decode_static.restype = ci
         L.mqa_append_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, sz, vp]
         L.mqa_append_decode.restype = ci
+        L.mqa_decode_grouped.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, sz, vp]
+        L.mqa_decode_grouped.restype = ci
+        L.mqa_decode_grouped_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
+        L.mqa_decode_grouped_workspace_bytes.restype = sz
         L.mqa_debug_schedule.argtypes = [vp, ci, ci, ci, ci, ci, vp, ci]; L.mqa_debug_schedule.restype = ci
         _lib = L
     return _lib
@@ -199,6 +203,27 @@ def mqa_append_decode(q, k_new, v_new, k_cache, v_cache, lengths, out, scale: fl
                                  float(scale), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "mqa_append_decode")
     return out
+
+
+def mqa_decode_grouped(q, k_cache, v_cache, lengths, out, scale: float, workspace=None, stream=None):
+    """Grouped-query / multihead decode: k_cache, v_cache are [B, KVH, Lmax, D]; q, out are [B, H, D]."""
+    B, H, D = q.shape
+    KVH, Lmax = k_cache.shape[1], k_cache.shape[2]
+    assert k_cache.shape == (B, KVH, Lmax, D) and v_cache.shape == k_cache.shape
+    assert lengths.shape == (B,) and out.shape == (B, H, D)
+    for t in (q, k_cache, v_cache, lengths, out):
+        assert t.is_cuda and t.is_contiguous()
+    if workspace is None:
+        n = int(lib().mqa_decode_grouped_workspace_bytes(B, H, KVH, D, Lmax))
+        if n == 0:
+            raise MqaError(MQA_ERR_UNSUPPORTED_SHAPE, "mqa_decode_grouped_workspace_bytes")
+        workspace = torch.empty(n, dtype=torch.uint8, device=q.device)
+        mqa_workspace_init(workspace, stream)
+    rc = lib().mqa_decode_grouped(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), lengths.data_ptr(),
+                                  out.data_ptr(), B, H, KVH, D, Lmax, float(scale),
+                                  workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "mqa_decode_grouped")
+    return out, workspace
 
 
 def mqa_check_status(workspace, stream=None) -> int:

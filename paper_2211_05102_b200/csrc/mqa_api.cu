@@ -98,7 +98,8 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* lengths, float* out,
                        int B, int H, int D, int Lmax, float scale,
                        const mqa_plan_t* plan,
-                       void* workspace, size_t workspace_bytes, void* stream, void* event_after_split)
+                       void* workspace, size_t workspace_bytes, void* stream, void* event_after_split,
+                       int kv_groups = 1)
 {
     if (!q || !k_cache || !v_cache || !lengths || !out || !workspace || !plan) return MQA_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || D <= 0 || Lmax <= 0) return MQA_ERR_INVALID_ARG;
@@ -125,7 +126,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.q = static_cast<const uint16_t*>(q);
     p.k = static_cast<const uint16_t*>(k_cache);
     p.v = static_cast<const uint16_t*>(v_cache);
-    p.lengths = lengths;
+    p.lengths = mqa::LenView{lengths, kv_groups};
     p.out = out;
     p.B = B; p.H = H; p.D = D; p.Lmax = Lmax;
     p.scale_log2 = scale * 1.4426950408889634f;
@@ -218,6 +219,31 @@ int mqa_append_decode(const void* q, const void* k_new, const void* v_new,
     return rc;
 }
 
+int mqa_decode_grouped(const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* lengths, float* out,
+                       int B, int H, int KVH, int D, int Lmax, float scale,
+                       void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (KVH <= 0 || H <= 0 || B <= 0) return MQA_ERR_INVALID_ARG;
+    if (H % KVH != 0) return MQA_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)B * KVH >= (1ll << 31)) return MQA_ERR_UNSUPPORTED_SHAPE;
+    // Each (sequence, key/value head) pair is one multiquery problem: H/KVH query heads sharing one K/V head
+    // over rows [0, lengths[b]).  With the caches laid out [B, KVH, Lmax, D] and q/out as [B, H, D] (the heads
+    // of a group adjacent) that is mqa_decode on B*KVH sequences, the lengths read through a grouped view.
+    const int Bg = B * KVH, Hg = H / KVH;
+    mqa_plan_t plan;
+    const int rc = mqa_decode_plan(Bg, Hg, D, Lmax, MQA_PATH_AUTO, &plan);
+    if (rc != MQA_OK) return rc;
+    return decode_impl(q, k_cache, v_cache, lengths, out, Bg, Hg, D, Lmax, scale, &plan,
+                       workspace, workspace_bytes, stream, nullptr, KVH);
+}
+
+size_t mqa_decode_grouped_workspace_bytes(int B, int H, int KVH, int D, int Lmax)
+{
+    if (KVH <= 0 || H <= 0 || B <= 0 || H % KVH != 0 || (long long)B * KVH >= (1ll << 31)) return 0;
+    return mqa_decode_workspace_bytes(B * KVH, H / KVH, D, Lmax);
+}
+
 int mqa_check_status(void* workspace, void* stream)
 {
     if (!workspace) return MQA_ERR_INVALID_ARG;
@@ -299,7 +325,7 @@ int mqa_debug_schedule(const int32_t* lengths_host, int B, int Lmax, int tile_ro
         prefix += nt;
     }
     mqa::SegmentWalker w;
-    w.init(lengths_host, B, Lmax, shift, (int)T, num_ctas, cta, b0, p0);
+    w.init(mqa::LenView{lengths_host, 1}, B, Lmax, shift, (int)T, num_ctas, cta, b0, p0);
     int n = 0;
     for (; !w.done(); w.next()) {
         if (n < max_segments) {

@@ -50,11 +50,19 @@ __host__ __device__ inline size_t workspace_bytes(int B, int H, int D) {
     return slots_offset(B) + (size_t)2 * kMaxCtas * slot_floats(H, D) * sizeof(float);
 }
 
+// Lengths as the kernels see them: entry b of a batch of B*kv_groups "sequences" is lengths[b / kv_groups]
+// (every key/value head of a sequence has that sequence's length); kv_groups = 1 for multiquery attention.
+struct LenView {
+    const int32_t* ptr;
+    int groups;
+    __host__ __device__ __forceinline__ int operator[](int b) const { return groups == 1 ? ptr[b] : ptr[b / groups]; }
+};
+
 struct Params {
     const uint16_t* q;        // bf16 bits [B,H,D]
     const uint16_t* k;        // [B,Lmax,D]
     const uint16_t* v;        // [B,Lmax,D]
-    const int32_t* lengths;   // [B]
+    LenView lengths;          // [B / kv_groups] int32, viewed per (sequence, key/value head)
     float* out;               // [B,H,D]
     int B, H, D, Lmax;
     float scale_log2;         // scale * log2(e): logits are kept in the base-2 domain
@@ -94,7 +102,7 @@ struct SchedShared {
 // Block-wide: total tile count T, and (b0, p0) for the tile `g0 = span_begin(cta)`.
 // Every thread returns T; sh.b0/sh.p0 are valid after the call when the run is non-empty.
 template <int NTHREADS>
-__device__ inline int schedule_prologue(const int32_t* __restrict__ lengths, int B, int Lmax,
+__device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
                                         int tile_shift, int G, int cta, SchedShared& sh)
 {
     const int tid = threadIdx.x;
@@ -142,14 +150,14 @@ __device__ inline int schedule_prologue(const int32_t* __restrict__ lengths, int
 
 // Walks the segments of one block's run.  All threads that use it hold identical state.
 struct SegmentWalker {
-    const int32_t* lengths;
+    LenView lengths;
     int Lmax, tile_shift, B;
     long long g0, g1;     // this block's run
     long long g;          // next tile to hand out
     int b, len, nt;       // current sequence
     long long P;          // global index of its first tile
 
-    __host__ __device__ void init(const int32_t* lengths_, int B_, int Lmax_, int tile_shift_, int T, int G,
+    __host__ __device__ void init(const LenView lengths_, int B_, int Lmax_, int tile_shift_, int T, int G,
                          int cta, int b0, int p0)
     {
         lengths = lengths_; B = B_; Lmax = Lmax_; tile_shift = tile_shift_;

@@ -96,7 +96,7 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     p.q = static_cast<const uint16_t*>(q);
     p.k = static_cast<const uint16_t*>(k_cache);
     p.v = static_cast<const uint16_t*>(v_cache);
-    p.lengths = lengths;
+    p.lengths = mqa::LenView{lengths, 1};
     p.out = out;
     p.B = B; p.H = H; p.D = D; p.Lmax = Lmax;
     p.scale_log2 = scale * 1.4426950408889634f;
