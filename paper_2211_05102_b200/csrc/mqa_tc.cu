@@ -27,7 +27,12 @@ namespace mqa {
 
 namespace {
 
-constexpr int kHeadsPerThread = 16;        // a softmax thread owns one cache row and 16 heads
+#ifndef MQA_HPT48
+#define MQA_HPT48 16
+#endif
+// Heads per softmax thread (a thread owns one cache row and this many heads): 16, or 24 for 48 heads
+// (two warpgroups instead of three: fewer threads in the named barrier and 170 instead of 128 registers).
+__host__ __device__ constexpr int heads_per_thread(int hp) { return hp == 48 ? MQA_HPT48 : 16; }
 constexpr int kTileShift = 7;
 constexpr int kTileRows = 128;
 constexpr int kSlotBytes = 16384;          // one ring slot: 128 rows x 64 cols (K) or 8192/D whole rows (V)
@@ -174,6 +179,39 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
           "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
         : "memory");
 }
+// 8 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7]))
+        : "memory");
+}
+// N = 16 or 24 consecutive columns.
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
+    static_assert(N == 8 || N == 16 || N == 24, "unsupported column count");
+    if (N == 8) { tmem_ld8(taddr, v); return; }
+    tmem_ld16(taddr, v);
+    if (N == 24) tmem_ld8(taddr + 16, v + 16);
+}
+template <int N>
+__device__ __forceinline__ void tmem_st(uint32_t taddr, const float* v) {
+    static_assert(N == 8 || N == 16 || N == 24, "unsupported column count");
+    if (N == 8) { tmem_st8(taddr, v); return; }
+    tmem_st16(taddr, v);
+    if (N == 24) tmem_st8(taddr + 16, v + 16);
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -197,18 +235,18 @@ __device__ __forceinline__ float warp_max_f32(float v) {
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-// Barrier over the softmax threads (named barrier 1) with an OR reduction of a flag.
-__device__ __forceinline__ bool softmax_bar_or(bool flag, int nthreads) {
+// Barrier over the 128 threads of one softmax warpgroup (named barrier 1 + group) with an OR reduction of a flag.
+__device__ __forceinline__ bool softmax_bar_or(bool flag, int bar_id) {
     uint32_t out, in = flag ? 1u : 0u;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, %2, p;\n\t"
+        "bar.red.or.pred q, %2, 128, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(out) : "r"(in), "r"(nthreads) : "memory");
+        : "=r"(out) : "r"(in), "r"(bar_id) : "memory");
     return out != 0;
 }
-__device__ __forceinline__ void softmax_bar_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
+__device__ __forceinline__ void softmax_bar_sync(int bar_id) { asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory"); }
 
 // Shared-memory matrix descriptors (sm_100 format), split into a constant high word (8-row groups 1024 B
 // apart, version 1, 128-byte swizzle) and a 32-bit low word (start address >> 4, leading offset >> 4), so
@@ -375,7 +413,8 @@ __device__ __forceinline__ void merge_sequence(const Params& p, int T, int b, in
 
 template <int D, int HP>
 struct TcLayout {
-    static constexpr int HG = HP / kHeadsPerThread;          // head groups = softmax warpgroups
+    static constexpr int HPT = heads_per_thread(HP);
+    static constexpr int HG = HP / HPT;                      // head groups = softmax warpgroups
     static constexpr int kSoftmaxThreads = 128 * HG;
     static constexpr int kThreads = 128 + kSoftmaxThreads;   // warps 0-3: producer, MMA issuer, two idle
     static constexpr int SPT = D / 64;            // ring slots per K tile and per V tile
@@ -720,13 +759,15 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         } else if (warp >= kSoftmaxWarp0) {
             // =============================== softmax + epilogue ===============================
             // Thread = (cache row of the tile, group of 16 heads).  Warp w reads tensor-memory lanes 32*(w%4)..+31.
-            constexpr int HPT = kHeadsPerThread;
-            constexpr int NSM = L::kSoftmaxThreads;
+            constexpr int HPT = L::HPT;
             const int ws = warp - kSoftmaxWarp0;
             const int wq = ws & 3;                              // lane quadrant
             const int hb = (ws >> 2) * HPT;                     // first head of this thread's group
             const int row = wq * 32 + lane;                     // cache row within the tile = tensor-memory lane
-            const int sid = tid - kSoftmaxWarp0 * 32;           // index among the softmax threads
+            const int gid = ws >> 2;                            // warpgroup = head group; the groups never synchronise with each other
+            const int NSM = 1 + gid;                            // this group's named barrier
+            const int hmine = hb + row;                         // the head this thread looks after in per-head bookkeeping (if row < HPT)
+            const bool leader = (gid == 0 && row == 0);
             const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
             TileCursor c;
             c.init(p, T, cta, misc.sched);
@@ -736,14 +777,14 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             int trace_n = (ws == 0) ? 0 : 100000; (void)trace_n;
             struct { bool valid, whole; int b, seg, slot_id, c_nt; long long c_P; float m_mine; } pend;
             pend.valid = false;
-            // Only the first softmax warp watches an mbarrier; the others are released through the named
-            // barrier, which also makes the outcome uniform across the group.
+            // Only the first warp of a warpgroup watches an mbarrier; the other three are released through the
+            // group's named barrier, which also makes the outcome uniform across the group.
             auto group_wait = [&](void* bar, uint32_t parity) -> bool {
 #ifdef MQA_GROUP_WAIT_ALL
                 return mbar_wait(bar, parity, abort_flag);
 #else
                 bool failed = false;
-                if (ws == 0) failed = !mbar_wait(bar, parity, abort_flag);
+                if (wq == 0) failed = !mbar_wait(bar, parity, abort_flag);
                 return !softmax_bar_or(failed, NSM);
 #endif
             };
@@ -760,13 +801,13 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 PROF_BEGIN();
                 float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, pend.slot_id);
                 const int Hp4 = round_up(H, 4);
-                if (!whole && sid < H) {
-                    slot_ptr[sid] = pend.m_mine;
-                    slot_ptr[Hp4 + sid] = misc.lsum[set][sid];
+                if (!whole && row < HPT && hmine < H) {
+                    slot_ptr[hmine] = pend.m_mine;
+                    slot_ptr[Hp4 + hmine] = misc.lsum[set][hmine];
                 }
                 float o[NACC][HPT];
 #pragma unroll
-                for (int j = 0; j < NACC; ++j) tmem_ld16(lane_base + kOCol + (uint32_t)(set * 128 + j * 64 + hb), o[j]);
+                for (int j = 0; j < NACC; ++j) tmem_ld<HPT>(lane_base + kOCol + (uint32_t)(set * 128 + j * 64 + hb), o[j]);
                 tmem_wait_ld();
                 tc_fence_before();
                 __syncwarp();
@@ -799,13 +840,14 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     // merges all of them after its own tiles are done (merge_sequence).
                     __threadfence();
                     softmax_bar_sync(NSM);
-                    if (sid == 0) {
+                    if (row == 0) {
+                        // every warpgroup of every block holding a part arrives once
                         const int i_first = cta_of_tile(pend.c_P, T, G), i_last = cta_of_tile(pend.c_P + pend.c_nt - 1, T, G);
                         const int nparts = (T >= G) ? (i_last - i_first + 1) : pend.c_nt;   // T < G: one tile per block
                         const int old = atomicAdd(ws_arrivals(p.workspace, p.B) + b, 1);
-                        if (old == nparts - 1) {
+                        if (old == nparts * L::HG - 1) {
                             __threadfence();
-                            const int k = misc.n_pending++;
+                            const int k = atomicAdd(&misc.n_pending, 1);
                             misc.pending[k] = b; misc.pending_p[k] = (int)pend.c_P; misc.pending_nt[k] = pend.c_nt;
                         }
                     }
@@ -826,7 +868,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 const int slot_id = c.w.seg_slot(cta);
                 const long long c_P = c.w.P;
                 const int c_nt = c.w.nt;
-                if (c.w.seg_owns_first_tile() && sid == 0) {
+                if (c.w.seg_owns_first_tile() && leader) {
                     SeqInfo si;
                     si.first_slot = whole ? -1 : slot_id;
                     si.last_cta = cta_of_tile(c.w.P + c.w.nt - 1, T, G);
@@ -834,7 +876,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 }
 #pragma unroll
                 for (int i = 0; i < HPT; ++i) l[i] = 0.f;
-                if (sid < HP) misc.m[sid] = -INFINITY;    // reference maximum per head, shared by all rows
+                if (row < HPT) misc.m[hmine] = -INFINITY;    // reference maximum per head, shared by all rows
                 softmax_bar_sync(NSM);
                 bool first = true;
                 for (;;) {
@@ -848,7 +890,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     TRACE(2, 30, ns);   // S ready
                     float y[HPT];
                     { PROF_BEGIN();
-                    tmem_ld16(lane_base + (uint32_t)(sb * 64 + hb), y);
+                    tmem_ld<HPT>(lane_base + (uint32_t)(sb * 64 + hb), y);
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
@@ -881,7 +923,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                             if (lane == i) misc.wred[wq][hb + i] = wm;
                         }
                         softmax_bar_sync(NSM);
-                        if (sid < HP) {
+                        if (row < HPT) {
+                            const int sid = hmine;
                             const float tm = fmaxf(fmaxf(misc.wred[0][sid], misc.wred[1][sid]), fmaxf(misc.wred[2][sid], misc.wred[3][sid]));
                             const float m_old = misc.m[sid];
                             const float m_new = fmaxf(m_old, tm);
@@ -899,11 +942,11 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                             for (int j = 0; j < NACC; ++j) {
                                 float o[HPT];
                                 const uint32_t ta = lane_base + kOCol + (uint32_t)((seg & 1) * 128 + j * 64 + hb);
-                                tmem_ld16(ta, o);
+                                tmem_ld<HPT>(ta, o);
                                 tmem_wait_ld();
 #pragma unroll
                                 for (int i = 0; i < HPT; ++i) o[i] *= misc.alpha[hb + i];
-                                tmem_st16(ta, o);
+                                tmem_st<HPT>(ta, o);
                             }
                             tmem_wait_st();
                             tc_fence_before();
@@ -969,7 +1012,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 // the pipeline here, the output is written after the first tile of the NEXT segment has been handed
                 // to the MMA issuer (the two segments use different accumulator sets in tensor memory).
                 TRACE(2, 40, ns);
-                pend.m_mine = (sid < HP) ? misc.m[sid] : 0.f;
+                pend.m_mine = (row < HPT) ? misc.m[hmine] : 0.f;
 #pragma unroll
                 for (int i = 0; i < HPT; ++i) {
                     float v = l[i];
@@ -978,7 +1021,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     if (lane == i) misc.wred[wq][hb + i] = v;
                 }
                 softmax_bar_sync(NSM);
-                if (sid < HP) misc.lsum[seg & 1][sid] = (misc.wred[0][sid] + misc.wred[1][sid]) + (misc.wred[2][sid] + misc.wred[3][sid]);
+                if (row < HPT) misc.lsum[seg & 1][hmine] = (misc.wred[0][hmine] + misc.wred[1][hmine]) + (misc.wred[2][hmine] + misc.wred[3][hmine]);
                 softmax_bar_sync(NSM);
                 pend.valid = true; pend.b = b; pend.seg = seg; pend.whole = whole; pend.slot_id = slot_id;
                 pend.c_P = c_P; pend.c_nt = c_nt;
