@@ -59,6 +59,7 @@ struct Barriers {
     unsigned long long s_full[4], s_empty[4];
     unsigned long long p_full[2], p_empty[2];
     unsigned long long o_full[2], o_empty[2];
+    unsigned long long merge;      // bulk copies of partial results into the idle ring
 };
 
 struct Misc {
@@ -329,16 +330,33 @@ struct SegIter {
 // K(0), .., K(lead), V(0), K(lead+1), V(1), ..., K(N-1), V(N-1-lead), .., V(N-1) with lead = kQkLead; every item fills
 // SPT consecutive slots.
 
+// Bulk copy global -> shared with completion on an mbarrier (addresses and size are multiples of 16 bytes).
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, void* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 // Log-sum-exp merge of the partial results of one cut sequence, by every thread of the block:
 //   M = max_s m_s;  out = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s
 // Parts are folded in block order with a running maximum, so the result does not depend on which
-// block performs the merge.  A thread owns GR float4 groups of the [H, D] output at a time and keeps the
-// loads of PU parts in flight together (the merge is bound by round trips to L2, not by bytes).
-template <int D, int GR, int PU>
-__device__ __forceinline__ void merge_parts(const Params& p, int T, int b, int i_first, int first_slot, int last_cta, int nthreads)
+// block performs the merge.  The merge is bound by round trips to L2, not by bytes, so the parts are not
+// read with a chain of loads: one thread bulk-copies as many whole slots as fit into the (now idle) K/V ring
+// at once, and every thread folds its float4 groups of the [H, D] output from shared memory.
+// Block-uniform; returns false when the bounded wait for the copies ran out.
+template <int D>
+__device__ __forceinline__ bool merge_sequence(const Params& p, int T, int b, int P, int nt, int nthreads,
+                                               unsigned char* stage, int stage_bytes, void* bar, uint32_t& phase,
+                                               volatile int* abort_flag)
 {
+    constexpr int GR = 7;                              // float4 groups per thread and pass (one pass covers H <= 64, D <= 256)
     const int H = p.H, G = p.num_ctas, Hp4 = round_up(H, 4);
     const int total = H * D / 4;                       // float4 groups of the output
+    const uint32_t part_bytes = (uint32_t)(slot_floats(H, D) * sizeof(float));
+    const int per_batch = stage_bytes / (int)part_bytes;
+    // which blocks hold the parts follows from the schedule alone
+    const int i_first = cta_of_tile(P, T, G), last_cta = cta_of_tile((long long)P + nt - 1, T, G);
+    const int first_slot = ((long long)P == span_begin(i_first, T, G)) ? 2 * i_first : 2 * i_first + 1;
+    auto owns_tiles = [&](int i) { return i == i_first || T >= G || span_begin(i, T, G) != span_begin(i + 1, T, G); };
     for (int base = 0; base < total; base += nthreads * GR) {
         float M[GR], Ls[GR];
         float4 acc[GR];
@@ -346,44 +364,41 @@ __device__ __forceinline__ void merge_parts(const Params& p, int T, int b, int i
         for (int g = 0; g < GR; ++g) { M[g] = -INFINITY; Ls[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
         int i2 = i_first;
         while (i2 <= last_cta) {
-            const float* sp[PU];
-            int np = 0;
-#pragma unroll
-            for (int u = 0; u < PU; ++u) sp[u] = nullptr;
-#pragma unroll
-            for (int u = 0; u < PU; ++u) {
-                // next block in [i2, last_cta] that owns tiles
-                while (i2 <= last_cta && i2 > i_first && span_begin(i2, T, G) == span_begin(i2 + 1, T, G)) ++i2;
-                if (i2 <= last_cta) { sp[u] = ws_slot(p.workspace, p.B, H, D, i2 == i_first ? first_slot : 2 * i2); ++i2; ++np; }
-            }
-            float ms[PU][GR], ls[PU][GR];
-            float4 as[PU][GR];
-#pragma unroll
-            for (int u = 0; u < PU; ++u) {
-#pragma unroll
-                for (int g = 0; g < GR; ++g) {
-                    const int e = base + g * nthreads + (int)threadIdx.x;
-                    if (u < np && e < total) {
-                        const int h = (e * 4) / D;
-                        ms[u][g] = __ldcg(sp[u] + h);
-                        ls[u][g] = __ldcg(sp[u] + Hp4 + h);
-                        as[u][g] = __ldcg(reinterpret_cast<const float4*>(sp[u] + 2 * Hp4) + e);
-                    }
+            // one batch: the next per_batch parts, copied together
+            int nb = 0, i3 = i2;
+            while (nb < per_batch && i3 <= last_cta) { if (owns_tiles(i3)) ++nb; ++i3; }
+            __syncthreads();                           // the staging area is free (earlier batch, earlier sequence, the ring)
+            if (threadIdx.x == 0) {
+                asm volatile("fence.proxy.async.global;" ::: "memory");   // the parts were written with ordinary stores
+                mbar_expect_tx(bar, (uint32_t)nb * part_bytes);
+                int u = 0;
+                for (int i = i2; i < i3; ++i) {
+                    if (!owns_tiles(i)) continue;
+                    bulk_g2s(stage + (size_t)u * part_bytes, ws_slot(p.workspace, p.B, H, D, i == i_first ? first_slot : 2 * i),
+                             part_bytes, bar);
+                    ++u;
                 }
             }
-#pragma unroll
-            for (int u = 0; u < PU; ++u) {
+            i2 = i3;
+            const bool failed = !mbar_wait(bar, phase, abort_flag);
+            phase ^= 1;
+            if (__syncthreads_or(failed)) return false;
+            for (int u = 0; u < nb; ++u) {
+                const float* sp = reinterpret_cast<const float*>(stage + (size_t)u * part_bytes);
 #pragma unroll
                 for (int g = 0; g < GR; ++g) {
                     const int e = base + g * nthreads + (int)threadIdx.x;
-                    if (u < np && e < total) {
-                        const float m_new = fmaxf(M[g], ms[u][g]);
+                    if (e < total) {
+                        const int h = (e * 4) / D;
+                        const float ms = sp[h], ls = sp[Hp4 + h];
+                        const float4 as = reinterpret_cast<const float4*>(sp + 2 * Hp4)[e];
+                        const float m_new = fmaxf(M[g], ms);
                         const float wa = (M[g] == -INFINITY) ? 0.f : ex2_approx(M[g] - m_new);
-                        const float wb = ex2_approx(ms[u][g] - m_new);
+                        const float wb = ex2_approx(ms - m_new);
                         M[g] = m_new;
-                        Ls[g] = fmaf(wa, Ls[g], wb * ls[u][g]);
-                        acc[g].x = fmaf(wa, acc[g].x, wb * as[u][g].x); acc[g].y = fmaf(wa, acc[g].y, wb * as[u][g].y);
-                        acc[g].z = fmaf(wa, acc[g].z, wb * as[u][g].z); acc[g].w = fmaf(wa, acc[g].w, wb * as[u][g].w);
+                        Ls[g] = fmaf(wa, Ls[g], wb * ls);
+                        acc[g].x = fmaf(wa, acc[g].x, wb * as.x); acc[g].y = fmaf(wa, acc[g].y, wb * as.y);
+                        acc[g].z = fmaf(wa, acc[g].z, wb * as.z); acc[g].w = fmaf(wa, acc[g].w, wb * as.w);
                     }
                 }
             }
@@ -398,17 +413,8 @@ __device__ __forceinline__ void merge_parts(const Params& p, int T, int b, int i
             }
         }
     }
-}
-
-template <int D>
-__device__ __forceinline__ void merge_sequence(const Params& p, int T, int b, int P, int nt, int nthreads)
-{
-    const int G = p.num_ctas;
-    // which blocks hold the parts follows from the schedule alone
-    const int i_first = cta_of_tile(P, T, G), last_cta = cta_of_tile((long long)P + nt - 1, T, G);
-    const int first_slot = ((long long)P == span_begin(i_first, T, G)) ? 2 * i_first : 2 * i_first + 1;
-    merge_parts<D, 6, 1>(p, T, b, i_first, first_slot, last_cta, nthreads);
     if (threadIdx.x == 0) ws_arrivals(p.workspace, p.B)[b] = 0;   // ready for the next call
+    return true;
 }
 
 template <int D, int HP>
@@ -462,6 +468,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         for (int i = 0; i < 4; ++i) { mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32); }
         for (int i = 0; i < 2; ++i) { mbar_init(&bars.p_full[i], L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], L::kSoftmaxThreads / 32); }
+        mbar_init(&bars.merge, 1);
         misc.abort_flag = 0;
         misc.n_pending = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1036,8 +1043,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     if (!misc.abort_flag) {
         const int n_pending = misc.n_pending;
 #ifndef MQA_X_SKIP_MERGE
+        // the ring, the q buffers and the probability buffers are idle now: one staging area for the merge
+        const int stage_bytes = nslots * kSlotBytes + 2 * L::kQBytes + 2 * kPBufs * L::kPBytes;
+        uint32_t merge_phase = 0;
         for (int k = 0; k < n_pending; ++k)
-            merge_sequence<D>(p, T, misc.pending[k], misc.pending_p[k], misc.pending_nt[k], L::kThreads);
+            if (!merge_sequence<D>(p, T, misc.pending[k], misc.pending_p[k], misc.pending_nt[k], L::kThreads,
+                                   ring, stage_bytes, &bars.merge, merge_phase, abort_flag)) break;
 #else
         if (tid == 0) for (int k = 0; k < n_pending; ++k) ws_arrivals(p.workspace, p.B)[misc.pending[k]] = 0;
 #endif
