@@ -75,7 +75,8 @@ enum {
  */
 typedef struct {
     int path;        /* MQA_PATH_FMA or MQA_PATH_TC (AUTO only as a request)  */
-    int num_ctas;    /* 1 .. MQA_MAX_CTAS                                      */
+    int num_ctas;    /* 1 .. MQA_MAX_CTAS; the TC path runs min(num_ctas, SM count) blocks
+                        (its blocks wait for one another, so all must be resident) */
     int tile_rows;   /* cache rows per tile: 64 (FMA) or 128 (TC)              */
 } mqa_plan_t;
 

@@ -132,6 +132,9 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = tile_shift_of(plan->tile_rows);
     p.num_ctas = plan->num_ctas;
+    // The tensor-core kernel's blocks wait for one another (merge of cut sequences), so all of them must be
+    // resident at once: one block per SM at most.
+    if (plan->path == MQA_PATH_TC && p.num_ctas > sm_count_or_default()) p.num_ctas = sm_count_or_default();
     p.lo_max_len = 0x7fffffff;
     p.workspace = static_cast<unsigned char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -38,8 +38,8 @@ __host__ __device__ inline size_t slot_floats(int H, int D) {
     return (size_t)2 * round_up(H, 4) + (size_t)H * D;
 }
 __host__ __device__ inline size_t seqinfo_offset() { return kHeaderBytes; }
-// One arrival counter per sequence (tensor-core path: the block that delivers the last partial result of a
-// cut sequence merges them).  Zero between calls: the merging block resets it.
+// One arrival counter per sequence (tensor-core path: the blocks holding parts of a cut sequence merge it
+// together once all parts have arrived).  Zero between calls: the last block to leave the merge resets it.
 __host__ __device__ inline size_t arrivals_offset(int B) {
     return kHeaderBytes + ((size_t)B * sizeof(SeqInfo) + 255) / 256 * 256;
 }
@@ -97,6 +97,7 @@ struct SchedShared {
     int total;
     int b0;         // sequence that contains the first tile of this block's run
     int p0;         // global index of that sequence's first tile
+    long long g0, g1;   // this block's run of tiles [g0, g1)
 };
 
 // Block-wide: total tile count T, and (b0, p0) for the tile `g0 = span_begin(cta)`.
@@ -138,6 +139,7 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
     int prefix = sh.warp_sums[warp] + incl - local;   // tiles before this thread's first sequence
     if (T > 0) {
         const long long g0 = span_begin(cta, T, G);
+        if (tid == 0) { sh.g0 = g0; sh.g1 = span_begin(cta + 1, T, G); }
         for (int b = b_lo; b < b_hi; ++b) {
             const int nt = (clamp_len(lengths[b], Lmax) + tile_rows - 1) >> tile_shift;
             if (nt > 0 && (long long)prefix <= g0 && g0 < (long long)prefix + nt) { sh.b0 = b; sh.p0 = prefix; }
@@ -160,8 +162,14 @@ struct SegmentWalker {
     __host__ __device__ void init(const LenView lengths_, int B_, int Lmax_, int tile_shift_, int T, int G,
                          int cta, int b0, int p0)
     {
+        init_span(lengths_, B_, Lmax_, tile_shift_, span_begin(cta, T, G), span_begin(cta + 1, T, G), b0, p0);
+    }
+    // The same with the run [g0, g1) already known (the schedule prologue leaves it in shared memory).
+    __host__ __device__ void init_span(const LenView lengths_, int B_, int Lmax_, int tile_shift_,
+                                       long long g0_, long long g1_, int b0, int p0)
+    {
         lengths = lengths_; B = B_; Lmax = Lmax_; tile_shift = tile_shift_;
-        g0 = span_begin(cta, T, G); g1 = span_begin(cta + 1, T, G); g = g0;
+        g0 = g0_; g1 = g1_; g = g0;
         if (g0 < g1) {
             b = b0; P = p0;
             len = clamp_len(lengths[b], Lmax);

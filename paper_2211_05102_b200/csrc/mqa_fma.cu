@@ -38,7 +38,8 @@ mqa_fma_kernel(const Params p)
     float* sM = sS + (size_t)p.H * kSStride;
     float* sL = sM + kMaxHeads;
     float* sAlpha = sL + kMaxHeads;
-    SchedShared& sched = *reinterpret_cast<SchedShared*>(sAlpha + kMaxHeads);
+    // 8-byte aligned (the record holds 64-bit tile indices; the row stride above is odd): total() reserves the slack
+    SchedShared& sched = *reinterpret_cast<SchedShared*>((reinterpret_cast<uintptr_t>(sAlpha + kMaxHeads) + 7) & ~uintptr_t(7));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int H = p.H, cta = blockIdx.x, G = p.num_ctas;

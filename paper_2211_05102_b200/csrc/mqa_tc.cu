@@ -45,6 +45,10 @@ constexpr uint32_t kTmemCols = 512;        // 4 S buffers @0,64,128,192; accumul
 #ifndef MQA_QK_LEAD
 #define MQA_QK_LEAD 1
 #endif
+#ifndef MQA_MMA_UNROLL
+#define MQA_MMA_UNROLL 1                   // the issuer's per-slot loops stay rolled: the issue rate is far from a limit, code size is not
+#endif
+constexpr int kMmaUnroll = MQA_MMA_UNROLL;
 #ifndef MQA_P_BUFS
 #define MQA_P_BUFS 1
 #endif
@@ -59,7 +63,7 @@ struct Barriers {
     unsigned long long s_full[4], s_empty[4];
     unsigned long long p_full[2], p_empty[2];
     unsigned long long o_full[2], o_empty[2];
-    unsigned long long merge;      // bulk copies of partial results into the idle ring
+    unsigned long long pub[2];     // softmax warps -> publisher warp: the partial result in slot 2*cta + j is stored
 };
 
 struct Misc {
@@ -67,9 +71,9 @@ struct Misc {
     SchedShared sched;
     uint32_t tmem_base;
     int abort_flag;
-    int n_pending;                 // cut sequences whose last partial result this block delivered
-    int pending[2];                // (a block has at most two partial segments)
-    int pending_p[2], pending_nt[2];   // first global tile and tile count of those sequences
+#ifdef MQA_TC_PROFILE
+    unsigned long long prof_ts[8];
+#endif
     float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
     __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
     __align__(16) float alpha[kMaxHeads];  // rescale factors
@@ -85,9 +89,12 @@ struct Misc {
 #endif
 #define PROF_END(idx) do { if (blockIdx.x == MQA_PROF_BLOCK && (threadIdx.x == 0 || threadIdx.x == 32 || threadIdx.x == 128)) \
     atomicAdd(ws_header(p.workspace) + 16 + (idx), (int)(clock64() - prof_t0_)); } while (0)
+// per-block phase timestamps (globaltimer ns), dumped with the start/end times
+#define PROF_TS(i) do { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_) :: "memory"); misc.prof_ts[i] = t_; } while (0)
 #else
 #define PROF_BEGIN() do {} while (0)
 #define PROF_END(idx) do {} while (0)
+#define PROF_TS(i) do {} while (0)
 #endif
 // Optional event trace (compile with -DMQA_TC_TRACE=<block>): one elected thread per role appends
 // (event id, tile counter, clock) records for that block to the last, unused partial slot.
@@ -104,6 +111,11 @@ enum { kProfProdEmpty = 0, kProfMmaSEmpty, kProfMmaQFull, kProfMmaKFull, kProfMm
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -130,8 +142,16 @@ __device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
 #endif
 // Bounded wait.  Returns false (and raises the block's abort flag) when the limit is hit
 // or another role has already given up.
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+#ifndef MQA_WAIT_INLINE
+#define MQA_WAIT_INLINE 0
+#endif
+// The spinning part is one shared copy, not one per call site: the roles' loops stay small in the instruction cache.
+#if MQA_WAIT_INLINE
+__device__ __forceinline__
+#else
+__device__ __noinline__
+#endif
+bool mbar_wait_slow(void* bar, uint32_t parity, volatile int* abort_flag) {
     const long long t0 = clock64();
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -140,6 +160,10 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, volatile i
 #endif
         if ((spins & 63u) == 0u && (clock64() - t0 > kWaitLimitCycles || *abort_flag)) { *abort_flag = 1; return false; }
     }
+}
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -285,7 +309,7 @@ struct TileCursor {
     int t, t1;        // current tile and end tile within the sequence
     int seg;          // segment counter of this block
     __device__ void init(const Params& p, int T, int cta, const SchedShared& sh) {
-        w.init(p.lengths, p.B, p.Lmax, kTileShift, T, p.num_ctas, cta, sh.b0, sh.p0);
+        w.init_span(p.lengths, p.B, p.Lmax, kTileShift, sh.g0, sh.g1, sh.b0, sh.p0);
         seg = 0;
         if (!w.done()) { t = w.seg_t0(); t1 = w.seg_t1(); }
     }
@@ -311,7 +335,7 @@ struct SegIter {
     __device__ void load() { ti = 0; t0 = w.seg_t0(); nt_seg = w.seg_t1() - t0; len = w.len; }
     __device__ int nvalid() const { return min(kTileRows, len - ((t0 + ti) << kTileShift)); }   // valid rows of the current tile
     __device__ void init(const Params& p, int T, int cta, const SchedShared& sh) {
-        w.init(p.lengths, p.B, p.Lmax, kTileShift, T, p.num_ctas, cta, sh.b0, sh.p0);
+        w.init_span(p.lengths, p.B, p.Lmax, kTileShift, sh.g0, sh.g1, sh.b0, sh.p0);
         seg = 0; valid = !w.done();
         if (valid) load();
     }
@@ -330,91 +354,102 @@ struct SegIter {
 // K(0), .., K(lead), V(0), K(lead+1), V(1), ..., K(N-1), V(N-1-lead), .., V(N-1) with lead = kQkLead; every item fills
 // SPT consecutive slots.
 
-// Bulk copy global -> shared with completion on an mbarrier (addresses and size are multiples of 16 bytes).
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, void* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
+// The schedule's 64-bit divisions, out of line: they run a few times per block, and inlined they are a large
+// part of the kernel's code.
+__device__ __noinline__ int cta_of_tile_nl(long long g, int T, int G) { return cta_of_tile(g, T, G); }
+__device__ __noinline__ long long span_begin_nl(int i, int T, int G) { return span_begin(i, T, G); }
 
-// Log-sum-exp merge of the partial results of one cut sequence, by every thread of the block:
+// Log-sum-exp merge of the partial results of one cut sequence:
 //   M = max_s m_s;  out = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s
-// Parts are folded in block order with a running maximum, so the result does not depend on which
-// block performs the merge.  The merge is bound by round trips to L2, not by bytes, so the parts are not
-// read with a chain of loads: one thread bulk-copies as many whole slots as fit into the (now idle) K/V ring
-// at once, and every thread folds its float4 groups of the [H, D] output from shared memory.
-// Block-uniform; returns false when the bounded wait for the copies ran out.
+// Every block that holds one of the sequence's `nparts` parts merges an equal slice of the [H, D] output
+// (block number `u` of them the u-th slice) once all parts have arrived, so the work after the last arrival is one
+// slice per block whatever the number of parts.  Parts are folded in block order with a running maximum and
+// each output element by exactly one thread: the result does not depend on timing.  The merge is bound by
+// round trips to L2, not by bytes, so a thread keeps the loads of several parts and output groups in flight.
+// All threads of the block call this; the blocks of one launch are co-resident (cooperative launch).
 template <int D>
-__device__ __forceinline__ bool merge_sequence(const Params& p, int T, int b, int P, int nt, int nthreads,
-                                               unsigned char* stage, int stage_bytes, void* bar, uint32_t& phase,
-                                               volatile int* abort_flag)
+__device__ __noinline__ void merge_slice(const Params& p, int T, int b, long long P, int i_first, int first_slot, int u, int nparts, int nthreads)
 {
-    constexpr int GR = 7;                              // float4 groups per thread and pass (one pass covers H <= 64, D <= 256)
+    constexpr int PB = 4, EU = 2;
     const int H = p.H, G = p.num_ctas, Hp4 = round_up(H, 4);
     const int total = H * D / 4;                       // float4 groups of the output
-    const uint32_t part_bytes = (uint32_t)(slot_floats(H, D) * sizeof(float));
-    const int per_batch = stage_bytes / (int)part_bytes;
-    // which blocks hold the parts follows from the schedule alone
-    const int i_first = cta_of_tile(P, T, G), last_cta = cta_of_tile((long long)P + nt - 1, T, G);
-    const int first_slot = ((long long)P == span_begin(i_first, T, G)) ? 2 * i_first : 2 * i_first + 1;
-    auto owns_tiles = [&](int i) { return i == i_first || T >= G || span_begin(i, T, G) != span_begin(i + 1, T, G); };
-    for (int base = 0; base < total; base += nthreads * GR) {
-        float M[GR], Ls[GR];
-        float4 acc[GR];
+    const int e_lo = total * u / nparts, e_hi = total * (u + 1) / nparts;   // total <= 4096, u < nparts <= 592
+    // part s lives in the head slot of the s-th block that owns tiles of the sequence (the first part possibly in a tail slot)
+    auto part_ptr = [&](int s) -> const float* {
+        // T < G: one tile per block, and all of the arithmetic fits in 32 bits
+        const int blk = (T >= G) ? i_first + s : (((int)P + s + 1) * G + T - 1) / T - 1;
+        return ws_slot(p.workspace, p.B, H, D, s == 0 ? first_slot : 2 * blk);
+    };
+    // EU output groups per thread and pass, PB parts each: EU*PB independent 16-byte loads in flight
+    for (int e0 = e_lo + (int)threadIdx.x; e0 < e_hi; e0 += EU * nthreads) {
+        float M[EU], Ls[EU];
+        float4 acc[EU];
 #pragma unroll
-        for (int g = 0; g < GR; ++g) { M[g] = -INFINITY; Ls[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        int i2 = i_first;
-        while (i2 <= last_cta) {
-            // one batch: the next per_batch parts, copied together
-            int nb = 0, i3 = i2;
-            while (nb < per_batch && i3 <= last_cta) { if (owns_tiles(i3)) ++nb; ++i3; }
-            __syncthreads();                           // the staging area is free (earlier batch, earlier sequence, the ring)
-            if (threadIdx.x == 0) {
-                asm volatile("fence.proxy.async.global;" ::: "memory");   // the parts were written with ordinary stores
-                mbar_expect_tx(bar, (uint32_t)nb * part_bytes);
-                int u = 0;
-                for (int i = i2; i < i3; ++i) {
-                    if (!owns_tiles(i)) continue;
-                    bulk_g2s(stage + (size_t)u * part_bytes, ws_slot(p.workspace, p.B, H, D, i == i_first ? first_slot : 2 * i),
-                             part_bytes, bar);
-                    ++u;
+        for (int k = 0; k < EU; ++k) { M[k] = -INFINITY; Ls[k] = 0.f; acc[k] = make_float4(0.f, 0.f, 0.f, 0.f); }
+        for (int s0 = 0; s0 < nparts; s0 += PB) {
+            float ms[EU][PB], ls[EU][PB];
+            float4 as[EU][PB];
+#pragma unroll
+            for (int i = 0; i < PB; ++i) {
+                if (s0 + i < nparts) {
+                    const float* sp = part_ptr(s0 + i);
+#pragma unroll
+                    for (int k = 0; k < EU; ++k) {
+                        const int e = e0 + k * nthreads;
+                        if (e < e_hi) {
+                            const int h = (e * 4) / D;
+                            ms[k][i] = __ldcg(sp + h);
+                            ls[k][i] = __ldcg(sp + Hp4 + h);
+                            as[k][i] = __ldcg(reinterpret_cast<const float4*>(sp + 2 * Hp4) + e);
+                        }
+                    }
                 }
             }
-            i2 = i3;
-            const bool failed = !mbar_wait(bar, phase, abort_flag);
-            phase ^= 1;
-            if (__syncthreads_or(failed)) return false;
-            for (int u = 0; u < nb; ++u) {
-                const float* sp = reinterpret_cast<const float*>(stage + (size_t)u * part_bytes);
 #pragma unroll
-                for (int g = 0; g < GR; ++g) {
-                    const int e = base + g * nthreads + (int)threadIdx.x;
-                    if (e < total) {
-                        const int h = (e * 4) / D;
-                        const float ms = sp[h], ls = sp[Hp4 + h];
-                        const float4 as = reinterpret_cast<const float4*>(sp + 2 * Hp4)[e];
-                        const float m_new = fmaxf(M[g], ms);
-                        const float wa = (M[g] == -INFINITY) ? 0.f : ex2_approx(M[g] - m_new);
-                        const float wb = ex2_approx(ms - m_new);
-                        M[g] = m_new;
-                        Ls[g] = fmaf(wa, Ls[g], wb * ls);
-                        acc[g].x = fmaf(wa, acc[g].x, wb * as.x); acc[g].y = fmaf(wa, acc[g].y, wb * as.y);
-                        acc[g].z = fmaf(wa, acc[g].z, wb * as.z); acc[g].w = fmaf(wa, acc[g].w, wb * as.w);
+            for (int i = 0; i < PB; ++i) {
+                if (s0 + i < nparts) {
+#pragma unroll
+                    for (int k = 0; k < EU; ++k) {
+                        if (e0 + k * nthreads < e_hi) {
+                            const float m_new = fmaxf(M[k], ms[k][i]);
+                            const float wa = (M[k] == -INFINITY) ? 0.f : ex2_approx(M[k] - m_new);
+                            const float wb = ex2_approx(ms[k][i] - m_new);
+                            M[k] = m_new;
+                            Ls[k] = fmaf(wa, Ls[k], wb * ls[k][i]);
+                            acc[k].x = fmaf(wa, acc[k].x, wb * as[k][i].x); acc[k].y = fmaf(wa, acc[k].y, wb * as[k][i].y);
+                            acc[k].z = fmaf(wa, acc[k].z, wb * as[k][i].z); acc[k].w = fmaf(wa, acc[k].w, wb * as[k][i].w);
+                        }
                     }
                 }
             }
         }
 #pragma unroll
-        for (int g = 0; g < GR; ++g) {
-            const int e = base + g * nthreads + (int)threadIdx.x;
-            if (e < total) {
-                const float inv = __frcp_rn(Ls[g]);
+        for (int k = 0; k < EU; ++k) {
+            const int e = e0 + k * nthreads;
+            if (e < e_hi) {
+                const float inv = __frcp_rn(Ls[k]);
                 reinterpret_cast<float4*>(p.out + (size_t)b * H * D)[e] =
-                    make_float4(acc[g].x * inv, acc[g].y * inv, acc[g].z * inv, acc[g].w * inv);
+                    make_float4(acc[k].x * inv, acc[k].y * inv, acc[k].z * inv, acc[k].w * inv);
             }
         }
     }
-    if (threadIdx.x == 0) ws_arrivals(p.workspace, p.B)[b] = 0;   // ready for the next call
-    return true;
+}
+
+// Zero rows [first, 8192/D) of a staged V slot (D/64 boxes of [rows x 128 B]); called by a whole warp.  Rare
+// (only a sequence's last tile has invalid rows), so it is kept out of line.
+template <int D>
+__device__ __noinline__ void zero_v_rows(unsigned char* slot_base, int first, int lane)
+{
+    constexpr int VR = 8192 / D;
+    for (int lr = first + lane; lr < VR; lr += 32) {
+        for (int cb = 0; cb < D / 64; ++cb) {
+            uint4* dst = reinterpret_cast<uint4*>(slot_base + cb * (VR * 128) + lr * 128);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0, 0, 0, 0);
+        }
+    }
+    fence_proxy_async();
+    __syncwarp();
 }
 
 template <int D, int HP>
@@ -428,12 +463,17 @@ struct TcLayout {
     static constexpr int VROWS = 8192 / D;        // cache rows per V slot: a slot is VROWS full rows, contiguous in global memory
     static constexpr int kQBytes = HP * D * 2;    // one q buffer: D/64 chunks of [HP rows x 128 B]
     static constexpr int kPBytes = 128 * 128;     // one probability buffer: 128 cache rows x 128 B (up to 64 heads)
-    static constexpr int kFixed = 2 * kQBytes + 2 * kPBufs * kPBytes + (int)sizeof(Misc);   // q x2, (hi, lo) x kPBufs
+#ifdef MQA_X_NOLO
+    static constexpr int kPHalves = 1;
+#else
+    static constexpr int kPHalves = 2;
+#endif
+    static constexpr int kFixed = 2 * kQBytes + kPHalves * kPBufs * kPBytes + (int)sizeof(Misc);   // q x2, (hi, lo) x kPBufs
     static int slots_for(int smem_limit) {
-        int n = (smem_limit - 1024 - kFixed) / kSlotBytes;
+        int n = (smem_limit - kFixed) / kSlotBytes;
         return n > kMaxSlots ? kMaxSlots : n;
     }
-    static int smem_bytes(int nslots) { return 1024 + nslots * kSlotBytes + kFixed; }
+    static int smem_bytes(int nslots) { return nslots * kSlotBytes + kFixed; }
 };
 
 template <int D, int HP>
@@ -443,12 +483,16 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 {
     using L = TcLayout<D, HP>;
     constexpr int SPT = L::SPT, NACC = L::NACC;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* ring = smem;
+    // Swizzled tiles need 1024-byte alignment; the dynamic segment is declared with it (no slack is reserved).
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    if (smem_u32(smem_raw) & 1023u) {   // block-uniform; nothing has been set up yet
+        if (threadIdx.x == 0) atomicExch(ws_header(p.workspace) + kHdrStatus, 3 /* MQA_ERR_MISALIGNED */);
+        return;
+    }
+    unsigned char* ring = smem_raw;
     unsigned char* q_buf = ring + (size_t)nslots * kSlotBytes;       // 2 buffers
     unsigned char* p_buf = q_buf + 2 * L::kQBytes;                   // 2 buffers of (hi, lo)
-    Misc& misc = *reinterpret_cast<Misc*>(p_buf + 2 * kPBufs * L::kPBytes);
+    Misc& misc = *reinterpret_cast<Misc*>(p_buf + L::kPHalves * kPBufs * L::kPBytes);
     Barriers& bars = misc.bars;
     volatile int* abort_flag = &misc.abort_flag;
 
@@ -468,9 +512,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         for (int i = 0; i < 4; ++i) { mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32); }
         for (int i = 0; i < 2; ++i) { mbar_init(&bars.p_full[i], L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], L::kSoftmaxThreads / 32); }
-        mbar_init(&bars.merge, 1);
+        for (int i = 0; i < 2; ++i) mbar_init(&bars.pub[i], L::kSoftmaxThreads / 32);
         misc.abort_flag = 0;
-        misc.n_pending = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -486,7 +529,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         ws_header(p.workspace)[kHdrTotalTiles] = T;
         ws_header(p.workspace)[kHdrNumCtas] = G;
     }
-    const int N = (T > 0) ? (int)(span_begin(cta + 1, T, G) - span_begin(cta, T, G)) : 0;   // tiles of this block
+    const int N = (T > 0) ? (int)(misc.sched.g1 - misc.sched.g0) : 0;   // tiles of this block
+    if (tid == 0) PROF_TS(1);
     // Empty sequences own no tile: their output rows are zeroed here, round-robin over the blocks.
     for (int b = cta; b < p.B; b += G) {
         if (clamp_len(p.lengths[b], p.Lmax) == 0) {
@@ -593,6 +637,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 if (ok && n >= kQkLead) { load_v(cv); cv.advance(); }
             }
             PROF_END(kProfProdTotal);
+            if (lane == 0) PROF_TS(2);
             if (!ok) {
                 // give copies already in flight a bounded chance to land before the block retires
                 for (int s = max(0, slot_seq - nslots); s < slot_seq; ++s) {
@@ -636,7 +681,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 const uint32_t qlo = q_lo + (uint32_t)(qb * (L::kQBytes >> 4));
                 const bool last = iq.last();
                 TRACE(1, 10, nq);   // QK: s_empty and q ready
-#pragma unroll
+#pragma unroll kMmaUnroll
                 for (int ch = 0; ch < SPT; ++ch) {
                     const int slot = cslot;
 #ifndef MQA_X_NOCHUNKSYNC
@@ -687,7 +732,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 const bool last = iv.last();
                 const bool use_lo = iv.len <= p.lo_max_len;
                 const int nvalid = iv.nvalid();
-#pragma unroll
+#pragma unroll kMmaUnroll
                 for (int vi = 0; vi < SPT; ++vi) {
                     constexpr int kStep = 2048 >> 4;               // 16 cache rows of 128 B
                     constexpr int VR = L::VROWS;                   // rows of this slot: [vi*VR, vi*VR + VR)
@@ -702,16 +747,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         // Rows beyond the sequence may hold any bits (0 * NaN would poison the accumulator): zero them
                         // in the staged tile.  This warp consumes the ring strictly in order, so the slot is known to
                         // hold this tile.
-                        for (int lr = max(0, nvalid - vi * VR) + lane; lr < VR; lr += 32) {
-#pragma unroll
-                            for (int cb = 0; cb < D / 64; ++cb) {
-                                uint4* dst = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + cb * (VR * 128) + lr * 128);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0, 0, 0, 0);
-                            }
-                        }
-                        fence_proxy_async();
-                        __syncwarp();
+                        zero_v_rows<D>(ring + (size_t)slot * kSlotBytes, max(0, nvalid - vi * VR), lane);
                     }
                     tc_fence_after();
                     TRACE(1, 21 + vi, np);   // V slot landed
@@ -763,6 +799,31 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             }
 #endif
             PROF_END(kProfMmaTotal);
+            if (lane == 0) PROF_TS(3);
+        } else if (warp == 2) {
+            // =============================== publisher of partial results ===============================
+            // A block has at most two partial segments (the head of its run in slot 2*cta, the tail in 2*cta+1).
+            // Once every softmax warp has stored its share of a slot, this warp makes the slot visible device-wide
+            // and counts the block's arrival for that sequence (the blocks merge a cut sequence together once all
+            // its parts have arrived).  Keeping the fence and the atomic here keeps them off the softmax warps.
+            SegmentWalker w;
+            w.init_span(p.lengths, p.B, p.Lmax, kTileShift, misc.sched.g0, misc.sched.g1, misc.sched.b0, misc.sched.p0);
+            while (!w.done()) {
+                if (!w.seg_is_whole()) {
+                    if (!mbar_wait(&bars.pub[w.seg_slot(cta) & 1], 0, abort_flag)) break;
+                    if (lane == 0) {
+                        const int i_first = cta_of_tile_nl(w.P, T, G), i_last = cta_of_tile_nl(w.P + w.nt - 1, T, G);
+                        const int nparts = (T >= G) ? (i_last - i_first + 1) : w.nt;   // T < G: one tile per block
+                        __threadfence();
+                        // counts to nparts as the parts arrive and on to 2*nparts as the blocks leave the merge; the
+                        // last increment wraps it to zero for the next call, so nobody needs the returned value
+                        atomicInc(reinterpret_cast<unsigned*>(ws_arrivals(p.workspace, p.B) + w.b), 2u * (unsigned)nparts - 1u);
+                    }
+                    __syncwarp();
+                }
+                w.next();
+            }
+            if (lane == 0) PROF_TS(5);
         } else if (warp >= kSoftmaxWarp0) {
             // =============================== softmax + epilogue ===============================
             // Thread = (cache row of the tile, group of 16 heads).  Warp w reads tensor-memory lanes 32*(w%4)..+31.
@@ -774,7 +835,6 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             const int gid = ws >> 2;                            // warpgroup = head group; the groups never synchronise with each other
             const int NSM = 1 + gid;                            // this group's named barrier
             const int hmine = hb + row;                         // the head this thread looks after in per-head bookkeeping (if row < HPT)
-            const bool leader = (gid == 0 && row == 0);
             const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
             TileCursor c;
             c.init(p, T, cta, misc.sched);
@@ -782,7 +842,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             bool ok = true;
             float l[HPT];
             int trace_n = (ws == 0) ? 0 : 100000; (void)trace_n;
-            struct { bool valid, whole; int b, seg, slot_id, c_nt; long long c_P; float m_mine; } pend;
+            struct { bool valid, whole; int b, seg, slot_id; float m_mine; } pend;
             pend.valid = false;
             // Only the first warp of a warpgroup watches an mbarrier; the other three are released through the
             // group's named barrier, which also makes the outcome uniform across the group.
@@ -843,21 +903,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                         for (int i = 0; i < HPT; ++i)
                             if (hb + i < H) dst[(size_t)i * D] = o[j][i];
                     }
-                    // Publish this partial result.  The block that delivers a sequence's last partial result
-                    // merges all of them after its own tiles are done (merge_sequence).
-                    __threadfence();
-                    softmax_bar_sync(NSM);
-                    if (row == 0) {
-                        // every warpgroup of every block holding a part arrives once
-                        const int i_first = cta_of_tile(pend.c_P, T, G), i_last = cta_of_tile(pend.c_P + pend.c_nt - 1, T, G);
-                        const int nparts = (T >= G) ? (i_last - i_first + 1) : pend.c_nt;   // T < G: one tile per block
-                        const int old = atomicAdd(ws_arrivals(p.workspace, p.B) + b, 1);
-                        if (old == nparts * L::HG - 1) {
-                            __threadfence();
-                            const int k = atomicAdd(&misc.n_pending, 1);
-                            misc.pending[k] = b; misc.pending_p[k] = (int)pend.c_P; misc.pending_nt[k] = pend.c_nt;
-                        }
-                    }
+                    // Hand the slot to the publisher warp, which makes it visible device-wide and counts the arrival;
+                    // this group goes straight on with its next tile.
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.pub[pend.slot_id & 1]);
                 }
                 TRACE(2, 43, pend.seg);
                 PROF_END(kProfSmEpilogue);
@@ -873,14 +922,6 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 const bool whole = c.w.seg_is_whole();
                 const bool use_lo = c.w.len <= p.lo_max_len;
                 const int slot_id = c.w.seg_slot(cta);
-                const long long c_P = c.w.P;
-                const int c_nt = c.w.nt;
-                if (c.w.seg_owns_first_tile() && leader) {
-                    SeqInfo si;
-                    si.first_slot = whole ? -1 : slot_id;
-                    si.last_cta = cta_of_tile(c.w.P + c.w.nt - 1, T, G);
-                    ws_seqinfo(p.workspace)[b] = si;
-                }
 #pragma unroll
                 for (int i = 0; i < HPT; ++i) l[i] = 0.f;
                 if (row < HPT) misc.m[hmine] = -INFINITY;    // reference maximum per head, shared by all rows
@@ -1031,28 +1072,66 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 if (row < HPT) misc.lsum[seg & 1][hmine] = (misc.wred[0][hmine] + misc.wred[1][hmine]) + (misc.wred[2][hmine] + misc.wred[3][hmine]);
                 softmax_bar_sync(NSM);
                 pend.valid = true; pend.b = b; pend.seg = seg; pend.whole = whole; pend.slot_id = slot_id;
-                pend.c_P = c_P; pend.c_nt = c_nt;
             }
             if (ok && pend.valid) ok = run_epilogue();
             PROF_END(kProfSmTotal);
+            if (ws == 0 && lane == 0) PROF_TS(4);
         }
     }
 
     __syncwarp();
     __syncthreads();
-    if (!misc.abort_flag) {
-        const int n_pending = misc.n_pending;
+    // ---------------- merge of the cut sequences ----------------
+    // Each block merges its slice of every cut sequence it holds a part of (at most two: the head and the tail
+    // of its run) after all parts of that sequence have arrived.  One thread watches the arrival counter with
+    // a bounded wait.  The counter runs on to 2*nparts as the blocks leave; the last one out zeroes it for the
+    // next call.
 #ifndef MQA_X_SKIP_MERGE
-        // the ring, the q buffers and the probability buffers are idle now: one staging area for the merge
-        const int stage_bytes = nslots * kSlotBytes + 2 * L::kQBytes + 2 * kPBufs * L::kPBytes;
-        uint32_t merge_phase = 0;
-        for (int k = 0; k < n_pending; ++k)
-            if (!merge_sequence<D>(p, T, misc.pending[k], misc.pending_p[k], misc.pending_nt[k], L::kThreads,
-                                   ring, stage_bytes, &bars.merge, merge_phase, abort_flag)) break;
-#else
-        if (tid == 0) for (int k = 0; k < n_pending; ++k) ws_arrivals(p.workspace, p.B)[misc.pending[k]] = 0;
-#endif
+    if (!misc.abort_flag && N > 0) {
+        struct Cut { int b, i_first, first_slot, u, nparts; long long P; };
+        Cut cut0 = {}, cut1 = {};
+        int ncut = 0;
+        SegmentWalker w;
+        w.init_span(p.lengths, p.B, p.Lmax, kTileShift, misc.sched.g0, misc.sched.g1, misc.sched.b0, misc.sched.p0);
+        for (; !w.done() && ncut < 2; w.next()) {
+            if (w.seg_is_whole()) continue;
+            const int i_first = cta_of_tile_nl(w.P, T, G), i_last = cta_of_tile_nl(w.P + w.nt - 1, T, G);
+            Cut c;
+            c.b = w.b; c.P = w.P; c.i_first = i_first;
+            c.first_slot = (w.P == span_begin_nl(i_first, T, G)) ? 2 * i_first : 2 * i_first + 1;
+            c.nparts = (T >= G) ? (i_last - i_first + 1) : w.nt;          // T < G: one tile per block
+            c.u = (T >= G) ? (cta - i_first) : (int)(w.g - w.P);          // this block's part number
+            if (ncut == 0) cut0 = c; else cut1 = c;
+            ++ncut;
+        }
+        if (ncut > 0) {
+            int* const counters = ws_arrivals(p.workspace, p.B);
+            bool failed = false;
+            if (tid == 0) {
+                const long long t0 = clock64();
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const Cut& ct = c == 0 ? cut0 : cut1;
+                    if (c < ncut && !failed)
+                        for (uint32_t spins = 1; ld_acquire_gpu(counters + ct.b) < ct.nparts; ++spins) {
+                            if (spins > 16u) __nanosleep(100);
+                            if ((spins & 63u) == 0u && clock64() - t0 > kWaitLimitCycles) { misc.abort_flag = 1; failed = true; break; }
+                        }
+                }
+            }
+            if (tid == 0) PROF_TS(6);
+            if (!__syncthreads_or(failed)) {
+                merge_slice<D>(p, T, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
+                if (ncut > 1) merge_slice<D>(p, T, cut1.b, cut1.P, cut1.i_first, cut1.first_slot, cut1.u, cut1.nparts, L::kThreads);
+                __syncthreads();   // every thread of this block has read its parts
+                if (tid == 0) {
+                    atomicInc(reinterpret_cast<unsigned*>(counters + cut0.b), 2u * (unsigned)cut0.nparts - 1u);
+                    if (ncut > 1) atomicInc(reinterpret_cast<unsigned*>(counters + cut1.b), 2u * (unsigned)cut1.nparts - 1u);
+                }
+            }
+        }
     }
+#endif
 #ifdef MQA_TC_PROFILE
     if (tid == 0) {
         unsigned long long ns1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
@@ -1063,7 +1142,9 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         // per-block start/end times and SM id, in the last (unused) partial slot
         unsigned long long* tl = reinterpret_cast<unsigned long long*>(ws_slot(p.workspace, p.B, p.H, D, 2 * kMaxCtas - 1));
         unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        tl[3 * blockIdx.x] = prof_ns0; tl[3 * blockIdx.x + 1] = ns1; tl[3 * blockIdx.x + 2] = smid;
+        misc.prof_ts[0] = prof_ns0; misc.prof_ts[7] = ns1;
+        for (int i = 0; i < 8; ++i) tl[9 * blockIdx.x + i] = misc.prof_ts[i];
+        tl[9 * blockIdx.x + 8] = smid;
     }
 #endif
     if (tid == 0 && misc.abort_flag) atomicExch(ws_header(p.workspace) + kHdrStatus, 7 /* MQA_ERR_TIMEOUT */);
@@ -1142,6 +1223,9 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
         e = cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
         if (e != cudaSuccess) return e;
         nslots = L::slots_for(smem_limit);
+#ifdef MQA_X_NSLOTS_ENV
+        if (const char* e2 = getenv("MQA_X_NSLOTS")) nslots = min(nslots, atoi(e2));
+#endif
         if (nslots < kMinSlots) return cudaErrorInvalidConfiguration;
         e = cudaFuncSetAttribute(mqa_tc_kernel<D, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::smem_bytes(nslots));
         if (e != cudaSuccess) return e;
@@ -1156,8 +1240,22 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
         }
         mc.q = p.q; mc.k = p.k; mc.v = p.v; mc.B = p.B; mc.H = p.H; mc.D = p.D; mc.Lmax = p.Lmax; mc.hp = HP;
     }
-    mqa_tc_kernel<D, HP><<<p.num_ctas, L::kThreads, L::smem_bytes(nslots), stream>>>(p, mc.mq, mc.mk, mc.mv, nslots);
-    return cudaGetLastError();
+    // Cooperative launch: the blocks wait for one another's partial results, so they must be co-resident
+    // (one block per SM, at most as many blocks as SMs).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.num_ctas);
+    cfg.blockDim = dim3((unsigned)L::kThreads);
+    cfg.dynamicSmemBytes = (size_t)L::smem_bytes(nslots);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+#ifdef MQA_X_COOP_ENV
+    if (const char* e3 = getenv("MQA_X_COOP")) cfg.numAttrs = atoi(e3);
+#endif
+    return cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
 }
 
 }  // namespace
