@@ -78,6 +78,10 @@ typedef struct {
     int num_ctas;    /* 1 .. MQA_MAX_CTAS; the TC path runs min(num_ctas, SM count) blocks
                         (its blocks wait for one another, so all must be resident) */
     int tile_rows;   /* cache rows per tile: 64 (FMA) or 128 (TC)              */
+    int adaptive;    /* TC path, 0 or 1: when every sequence of the batch owns the same
+                        number of tiles the kernel may share them among fewer blocks
+                        (mqa_uniform_ctas) so that the cuts fall on sequence boundaries;
+                        mqa_decode_plan sets it, 0 pins the block count to num_ctas */
 } mqa_plan_t;
 
 #define MQA_MAX_CTAS 592          /* upper bound on mqa_plan_t.num_ctas (4 per SM on 148 SMs) */
@@ -248,6 +252,22 @@ int mqa_last_launch_count(void);
 int mqa_decode_static(const void* q, const void* k_cache, const void* v_cache,
                       const int32_t* lengths, float* out,
                       int B, int H, int D, int Lmax, float scale, void* stream);
+
+/*
+ * Block count an adaptive plan uses for a batch in which each of the B sequences
+ * owns `tiles_per_sequence` K/V tiles, given the plan's num_ctas: the split-count
+ * heuristic for uniform batches (the paper fixes no split; Section 3.3 only
+ * states that the K/V cache load dominates decode attention).  With an even
+ * share of the flattened tiles almost every block boundary cuts a sequence, and
+ * each cut costs two partial epilogues and a merge.  A block count that divides
+ * B (whole sequences per block), or a multiple of B whose factor divides the
+ * tile count (every sequence in equal parts), avoids that and is chosen when
+ * the modelled slow-down of the K/V stream (fewer streaming SMs) stays below
+ * the modelled saving.  Returns num_ctas itself when no such count qualifies.
+ * Any other batch always runs on num_ctas blocks.  Host-only, no device is
+ * touched; returns a negated mqa_status_t for non-positive arguments.
+ */
+int mqa_uniform_ctas(int B, int tiles_per_sequence, int num_ctas);
 
 /*
  * Host replay of the device tile schedule, for tests and tooling (no device is

@@ -33,14 +33,17 @@ EXPORTS = [
     "mqa_status_string", "mqa_decode_workspace_bytes", "mqa_workspace_init", "mqa_decode_plan",
     "mqa_decode", "mqa_decode_with_plan", "mqa_decode_profiled", "mqa_check_status", "mqa_decode_host_scratch_bytes",
     "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static", "mqa_append_decode", "mqa_decode_grouped", "mqa_decode_grouped_workspace_bytes",
+    "mqa_uniform_ctas",
 ]
 
 
 class Plan(ctypes.Structure):
-    _fields_ = [("path", ctypes.c_int), ("num_ctas", ctypes.c_int), ("tile_rows", ctypes.c_int)]
+    _fields_ = [("path", ctypes.c_int), ("num_ctas", ctypes.c_int), ("tile_rows", ctypes.c_int),
+                ("adaptive", ctypes.c_int)]
 
     def __repr__(self):
-        return f"Plan(path={self.path}, num_ctas={self.num_ctas}, tile_rows={self.tile_rows})"
+        return (f"Plan(path={self.path}, num_ctas={self.num_ctas}, tile_rows={self.tile_rows}, "
+                f"adaptive={self.adaptive})")
 
 
 class MqaError(RuntimeError):
@@ -82,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_grouped_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
         L.mqa_decode_grouped_workspace_bytes.restype = sz
         L.mqa_debug_schedule.argtypes = [vp, ci, ci, ci, ci, ci, vp, ci]; L.mqa_debug_schedule.restype = ci
+        L.mqa_uniform_ctas.argtypes = [ci, ci, ci]; L.mqa_uniform_ctas.restype = ci
         _lib = L
     return _lib
 
@@ -245,6 +249,14 @@ def mqa_decode_host(q, k_cache, v_cache, lengths, out, scale: float, scratch, st
 
 def mqa_last_launch_count() -> int:
     return int(lib().mqa_last_launch_count())
+
+
+def mqa_uniform_ctas(B: int, tiles_per_sequence: int, num_ctas: int) -> int:
+    """Block count an adaptive plan uses for a batch of B sequences of equal tile count (host-only)."""
+    n = lib().mqa_uniform_ctas(B, tiles_per_sequence, num_ctas)
+    if n < 0:
+        raise MqaError(-n, "mqa_uniform_ctas")
+    return n
 
 
 def mqa_debug_schedule(lengths, Lmax: int, tile_rows: int, num_ctas: int, cta: int, max_segments: int = 4096):

@@ -91,6 +91,7 @@ int mqa_decode_plan(int B, int H, int D, int Lmax, int requested_path, mqa_plan_
     if (ctas > MQA_MAX_CTAS) ctas = MQA_MAX_CTAS;
     if (ctas < 1) ctas = 1;
     plan->num_ctas = (int)ctas;
+    plan->adaptive = (path == MQA_PATH_TC) ? 1 : 0;
     return MQA_OK;
 }
 
@@ -108,6 +109,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     if (plan->num_ctas < 1 || plan->num_ctas > MQA_MAX_CTAS) return MQA_ERR_INVALID_ARG;
     if (plan->path != MQA_PATH_FMA && plan->path != MQA_PATH_TC) return MQA_ERR_INVALID_ARG;
     if (plan->tile_rows != ((plan->path == MQA_PATH_TC) ? 128 : 64)) return MQA_ERR_INVALID_ARG;
+    if (plan->adaptive != 0 && plan->adaptive != 1) return MQA_ERR_INVALID_ARG;
     if (plan->path == MQA_PATH_TC && !mqa::tc_supported(H, D)) return MQA_ERR_UNSUPPORTED_SHAPE;
     if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) ||
         !aligned(lengths, 4) || !aligned(workspace, 256))
@@ -132,6 +134,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = tile_shift_of(plan->tile_rows);
     p.num_ctas = plan->num_ctas;
+    p.adaptive = (plan->path == MQA_PATH_TC) ? plan->adaptive : 0;
     // The tensor-core kernel's blocks wait for one another (merge of cut sequences), so all of them must be
     // resident at once: one block per SM at most.
     if (plan->path == MQA_PATH_TC && p.num_ctas > sm_count_or_default()) p.num_ctas = sm_count_or_default();
@@ -307,6 +310,12 @@ int mqa_decode_host(const void* q_host, const void* k_cache_host, const void* v_
 }
 
 int mqa_last_launch_count(void) { return g_last_launches; }
+
+int mqa_uniform_ctas(int B, int tiles_per_sequence, int num_ctas)
+{
+    if (B <= 0 || tiles_per_sequence <= 0 || num_ctas <= 0 || num_ctas > MQA_MAX_CTAS) return -MQA_ERR_INVALID_ARG;
+    return mqa::uniform_ctas(B, tiles_per_sequence, num_ctas);
+}
 
 int mqa_debug_schedule(const int32_t* lengths_host, int B, int Lmax, int tile_rows, int num_ctas, int cta,
                        int32_t* records, int max_segments)

@@ -67,7 +67,8 @@ struct Params {
     int B, H, D, Lmax;
     float scale_log2;         // scale * log2(e): logits are kept in the base-2 domain
     int tile_shift;           // log2(tile_rows)
-    int num_ctas;             // G
+    int num_ctas;             // G (an upper bound when `adaptive` is set)
+    int adaptive;             // tensor-core path: the kernel may run a uniform batch on fewer blocks (uniform_ctas)
     int lo_max_len;           // tensor-core path: sequences up to this length use hi+lo bf16 probabilities
     unsigned char* workspace;
 };
@@ -92,27 +93,62 @@ __host__ __device__ inline int cta_of_tile(long long g, int T, int G) {
     return (int)(((g + 1) * G + T - 1) / T) - 1;
 }
 
+// Block count for a batch in which every one of the B sequences owns the same number of tiles `nt`.
+// With G blocks sharing T = B*nt tiles evenly, almost every block boundary cuts a sequence, and each cut costs
+// two partial epilogues and a merge (about 8 us per block in total, measured).  A block count g whose cuts all
+// fall on sequence boundaries (g divides B: whole sequences per block) or cut every sequence into the same
+// number of equal parts (B divides g and g/B divides nt) avoids most of that; it is chosen when the K/V stream
+// is not slowed by more than the saving.  Stream model: one SM sustains a tile per kPerSmTileNs, and about
+// kSmsToSaturate of them saturate HBM, so fewer blocks than that stretch the stream proportionally.
+__host__ __device__ inline int uniform_ctas(int B, int nt, int G)
+{
+    constexpr float kPerSmTileNs = 2330.f, kSmsToSaturate = 123.f, kCutSavingNs = 7000.f;
+    const long long T = (long long)B * nt;
+    if (nt <= 0 || T <= G) return G;
+    auto stream_ns = [&](int g) { return (float)T * kPerSmTileNs / (g < kSmsToSaturate ? (float)g : kSmsToSaturate); };
+    int cand = 0;
+    if (B >= G) {
+        // whole sequences per block: the largest divisor of B that is <= G, if it is near G
+        const int k0 = (B + G - 1) / G;
+        for (int k = k0; k < k0 + 4 && cand == 0; ++k)
+            if (B % k == 0) cand = B / k;
+    } else {
+        // every sequence cut into s equal parts
+        const int s0 = G / B;
+        for (int s = s0; s >= 1 && s > s0 - 4 && cand == 0; --s)
+            if (nt % s == 0) cand = B * s;
+    }
+    if (cand <= 0 || cand >= G) return G;
+    return (stream_ns(cand) - stream_ns(G) < kCutSavingNs) ? cand : G;
+}
+
 struct SchedShared {
     int warp_sums[32];
     int total;
     int b0;         // sequence that contains the first tile of this block's run
     int p0;         // global index of that sequence's first tile
     long long g0, g1;   // this block's run of tiles [g0, g1)
+    int G;              // blocks that share the tiles (the launch's block count unless the plan is adaptive)
 };
 
 // Block-wide: total tile count T, and (b0, p0) for the tile `g0 = span_begin(cta)`.
 // Every thread returns T; sh.b0/sh.p0 are valid after the call when the run is non-empty.
 template <int NTHREADS>
 __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
-                                        int tile_shift, int G, int cta, SchedShared& sh)
+                                        int tile_shift, int G, int cta, SchedShared& sh, bool adaptive = false)
 {
     const int tid = threadIdx.x;
     const int tile_rows = 1 << tile_shift;
     const int per = (B + NTHREADS - 1) / NTHREADS;
     const int b_lo = min(B, tid * per), b_hi = min(B, b_lo + per);
     int local = 0;
-    for (int b = b_lo; b < b_hi; ++b)
-        local += (clamp_len(lengths[b], Lmax) + tile_rows - 1) >> tile_shift;
+    const int nt_first = adaptive ? (clamp_len(lengths[0], Lmax) + tile_rows - 1) >> tile_shift : 0;
+    bool uniform = adaptive;
+    for (int b = b_lo; b < b_hi; ++b) {
+        const int nt = (clamp_len(lengths[b], Lmax) + tile_rows - 1) >> tile_shift;
+        local += nt;
+        uniform = uniform && nt == nt_first;
+    }
     // inclusive scan within the warp
     int incl = local;
     const int lane = tid & 31, warp = tid >> 5;
@@ -122,7 +158,7 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
         if (lane >= o) incl += t;
     }
     if (lane == 31) sh.warp_sums[warp] = incl;
-    __syncthreads();
+    uniform = __syncthreads_and(uniform) != 0;
     if (warp == 0) {
         int w = (lane < NTHREADS / 32) ? sh.warp_sums[lane] : 0;
         int wi = w;
@@ -136,8 +172,10 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
     }
     __syncthreads();
     const int T = sh.total;
+    if (uniform) G = uniform_ctas(B, nt_first, G);    // identical in every thread of every block
+    if (tid == 0) sh.G = G;
     int prefix = sh.warp_sums[warp] + incl - local;   // tiles before this thread's first sequence
-    if (T > 0) {
+    if (T > 0 && cta < G) {
         const long long g0 = span_begin(cta, T, G);
         if (tid == 0) { sh.g0 = g0; sh.g1 = span_begin(cta + 1, T, G); }
         for (int b = b_lo; b < b_hi; ++b) {
@@ -145,6 +183,8 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
             if (nt > 0 && (long long)prefix <= g0 && g0 < (long long)prefix + nt) { sh.b0 = b; sh.p0 = prefix; }
             prefix += nt;
         }
+    } else if (tid == 0) {
+        sh.g0 = sh.g1 = 0;                            // a block beyond the chosen count owns no tiles
     }
     __syncthreads();
     return T;

@@ -102,6 +102,7 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = (plan.tile_rows == 128) ? 7 : 6;
     p.num_ctas = plan.num_ctas;
+    p.adaptive = (plan.path == MQA_PATH_TC) ? plan.adaptive : 0;
     p.lo_max_len = 0x7fffffff;
     p.workspace = ws;
     cudaError_t e = (plan.path == MQA_PATH_TC) ? mqa::launch_tc(p, st) : mqa::launch_fma(p, st);

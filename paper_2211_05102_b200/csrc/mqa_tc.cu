@@ -72,7 +72,7 @@ struct Misc {
     uint32_t tmem_base;
     int abort_flag;
 #ifdef MQA_TC_PROFILE
-    unsigned long long prof_ts[8];
+    unsigned long long prof_ts[12];
 #endif
     float wred[4][kMaxHeads];      // cross-warp exchange (tile maxima / row sums)
     __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
@@ -368,10 +368,10 @@ __device__ __noinline__ long long span_begin_nl(int i, int T, int G) { return sp
 // round trips to L2, not by bytes, so a thread keeps the loads of several parts and output groups in flight.
 // All threads of the block call this; the blocks of one launch are co-resident (cooperative launch).
 template <int D>
-__device__ __noinline__ void merge_slice(const Params& p, int T, int b, long long P, int i_first, int first_slot, int u, int nparts, int nthreads)
+__device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, long long P, int i_first, int first_slot, int u, int nparts, int nthreads)
 {
     constexpr int PB = 4, EU = 2;
-    const int H = p.H, G = p.num_ctas, Hp4 = round_up(H, 4);
+    const int H = p.H, Hp4 = round_up(H, 4);
     const int total = H * D / 4;                       // float4 groups of the output
     const int e_lo = total * u / nparts, e_hi = total * (u + 1) / nparts;   // total <= 4096, u < nparts <= 592
     // part s lives in the head slot of the s-th block that owns tiles of the sequence (the first part possibly in a tail slot)
@@ -502,7 +502,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     unsigned long long prof_ns0 = 0; long long prof_c0 = 0;
     if (tid == 0) { asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(prof_ns0)); prof_c0 = clock64(); }
 #endif
-    const int cta = blockIdx.x, G = p.num_ctas, H = p.H;
+    const int cta = blockIdx.x, H = p.H;
 
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
@@ -522,7 +522,9 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         tc_fence_before();
     }
-    const int T = schedule_prologue<L::kThreads>(p.lengths, p.B, p.Lmax, kTileShift, G, cta, misc.sched);   // has __syncthreads
+    const int T = schedule_prologue<L::kThreads>(p.lengths, p.B, p.Lmax, kTileShift, p.num_ctas, cta, misc.sched,
+                                                 p.adaptive != 0);   // has __syncthreads
+    const int G = misc.sched.G;   // blocks that share the tiles (fewer than launched for some uniform batches)
     tc_fence_after();
     const uint32_t tmem = misc.tmem_base;
     if (cta == 0 && tid == 0) {
@@ -532,7 +534,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     const int N = (T > 0) ? (int)(misc.sched.g1 - misc.sched.g0) : 0;   // tiles of this block
     if (tid == 0) PROF_TS(1);
     // Empty sequences own no tile: their output rows are zeroed here, round-robin over the blocks.
-    for (int b = cta; b < p.B; b += G) {
+    for (int b = cta; b < p.B; b += (int)gridDim.x) {
         if (clamp_len(p.lengths[b], p.Lmax) == 0) {
             float4* dst = reinterpret_cast<float4*>(p.out + (size_t)b * H * D);
             for (int i = tid; i < H * D / 4; i += L::kThreads) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1121,9 +1123,15 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             }
             if (tid == 0) PROF_TS(6);
             if (!__syncthreads_or(failed)) {
-                merge_slice<D>(p, T, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
-                if (ncut > 1) merge_slice<D>(p, T, cut1.b, cut1.P, cut1.i_first, cut1.first_slot, cut1.u, cut1.nparts, L::kThreads);
+                if (tid == 0) PROF_TS(8);
+                merge_slice<D>(p, T, G, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
+                if (ncut > 1) merge_slice<D>(p, T, G, cut1.b, cut1.P, cut1.i_first, cut1.first_slot, cut1.u, cut1.nparts, L::kThreads);
+                if (tid == 0) PROF_TS(9);
+#ifdef MQA_X_MERGE_TWICE
+                merge_slice<D>(p, T, G, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
+#endif
                 __syncthreads();   // every thread of this block has read its parts
+                if (tid == 0) PROF_TS(10);
                 if (tid == 0) {
                     atomicInc(reinterpret_cast<unsigned*>(counters + cut0.b), 2u * (unsigned)cut0.nparts - 1u);
                     if (ncut > 1) atomicInc(reinterpret_cast<unsigned*>(counters + cut1.b), 2u * (unsigned)cut1.nparts - 1u);
@@ -1143,8 +1151,8 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
         unsigned long long* tl = reinterpret_cast<unsigned long long*>(ws_slot(p.workspace, p.B, p.H, D, 2 * kMaxCtas - 1));
         unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
         misc.prof_ts[0] = prof_ns0; misc.prof_ts[7] = ns1;
-        for (int i = 0; i < 8; ++i) tl[9 * blockIdx.x + i] = misc.prof_ts[i];
-        tl[9 * blockIdx.x + 8] = smid;
+        for (int i = 0; i < 12; ++i) tl[13 * blockIdx.x + i] = misc.prof_ts[i];
+        tl[13 * blockIdx.x + 12] = smid;
     }
 #endif
     if (tid == 0 && misc.abort_flag) atomicExch(ws_header(p.workspace) + kHdrStatus, 7 /* MQA_ERR_TIMEOUT */);

@@ -55,5 +55,6 @@ def plans_for(B, H, D, Lmax, ctas=(None,)):
         except binding.MqaError:
             continue
         for c in ctas:
-            out.append(binding.Plan(base.path, base.num_ctas if c is None else c, base.tile_rows))
+            # None: the library's own plan (adaptive block count); a number pins the block count
+            out.append(base if c is None else binding.Plan(base.path, c, base.tile_rows))
     return out

@@ -148,3 +148,26 @@ def test_launch_count_is_reported():
     q, k, v, lengths = make_inputs(w)
     run_gpu(q, k, v, lengths, w.scale)
     assert binding.mqa_last_launch_count() >= 1
+
+
+@pytest.mark.parametrize("B,H,L", [(160, 16, 256), (50, 48, 512), (296, 8, 130), (64, 32, 1024)])
+def test_uniform_batches_under_the_adaptive_plan(B, H, L):
+    """Batches of equal tile count, where the library's own plan may share the tiles among fewer blocks than
+    it launches: same results as the pinned block count, and the block count the kernel reports is the
+    heuristic's."""
+    D, Lmax = 256, L + 40
+    lengths = [L - (i % 3) for i in range(B)]        # equal tile counts, unequal lengths
+    q, k, v, ln = make_custom(B, H, D, Lmax, seed=4242 + B, lengths=lengths)
+    k, v = poison_padding(k, v, ln, 0x7FC0)
+    expect = ref.mqa_decode_ref(q, k, v, ln, 1.0 / math.sqrt(D))
+    plan = binding.mqa_decode_plan(B, H, D, Lmax, binding.MQA_PATH_TC)
+    assert plan.adaptive == 1
+    ws = binding.alloc_workspace(B, H, D, Lmax)
+    got = run_gpu(q, k, v, ln, 1.0 / math.sqrt(D), plan=plan, workspace=ws)
+    assert_close(got, expect, f"adaptive B={B}")
+    nt = (L + 127) // 128
+    assert int(ws[:16].view(torch.int32)[3]) == binding.mqa_uniform_ctas(B, nt, plan.num_ctas)
+    pinned = binding.Plan(plan.path, plan.num_ctas, plan.tile_rows)
+    got2 = run_gpu(q, k, v, ln, 1.0 / math.sqrt(D), plan=pinned, workspace=ws)
+    assert_close(got2, expect, f"pinned B={B}")
+    assert int(ws[:16].view(torch.int32)[3]) == plan.num_ctas

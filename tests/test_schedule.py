@@ -67,3 +67,46 @@ def test_schedule_partitions_the_tiles(lengths, Lmax, tile, G):
         expect = [first_slot] + [2 * i for i in range(first_slot // 2 + 1, last_cta + 1)
                                  if spans[i][0] != spans[i][1]]
         assert [s for _, s in sorted(parts[b])] == expect
+
+
+def test_uniform_ctas_keeps_cuts_on_sequence_boundaries():
+    """The split-count heuristic for uniform batches: it never asks for more blocks than the plan has, and
+    whatever smaller count it picks either takes whole sequences per block or cuts every sequence into the
+    same number of equal parts."""
+    for B in list(range(1, 70)) + [96, 100, 128, 148, 200, 256, 296, 300, 444, 500, 512, 1000, 1024, 4096]:
+        for nt in (1, 2, 3, 4, 7, 8, 12, 16, 64, 256):
+            for G in (1, 7, 128, 132, 148, 592):
+                g = binding.mqa_uniform_ctas(B, nt, G)
+                assert 1 <= g <= G
+                if g != G:
+                    whole = B % g == 0
+                    equal_parts = g % B == 0 and nt % (g // B) == 0
+                    assert whole or equal_parts, (B, nt, G, g)
+                if B * nt <= G:
+                    assert g == G     # one tile per block: nothing to align
+
+
+def test_uniform_ctas_on_the_named_shapes():
+    # 512 sequences of 16 tiles on 148 SMs: 4 whole sequences per block
+    assert binding.mqa_uniform_ctas(512, 16, 148) == 128
+    # 64 sequences of 16 tiles: every sequence in two halves
+    assert binding.mqa_uniform_ctas(64, 16, 148) == 128
+    # no near divisor: the even share of the flattened tiles stays
+    assert binding.mqa_uniform_ctas(300, 8, 148) == 148
+    assert binding.mqa_uniform_ctas(200, 16, 148) == 148
+    with pytest.raises(binding.MqaError):
+        binding.mqa_uniform_ctas(0, 16, 148)
+
+
+@pytest.mark.parametrize("B,nt,G", [(512, 16, 148), (64, 16, 148), (160, 2, 148), (50, 4, 148), (32, 64, 148)])
+def test_aligned_block_count_has_no_ragged_cut(B, nt, G):
+    """Replay the schedule at the chosen block count: blocks hold whole sequences only, or every sequence is
+    cut into parts of equal size."""
+    g = binding.mqa_uniform_ctas(B, nt, G)
+    assert g < G
+    ln = torch.full((B,), nt * 128, dtype=torch.int32)
+    sizes = set()
+    for cta in range(g):
+        for (b, t0, t1, whole, slot, owns_first, last_cta) in binding.mqa_debug_schedule(ln, nt * 128, 128, g, cta):
+            sizes.add(t1 - t0)
+    assert len(sizes) == 1 and nt % sizes.pop() == 0
