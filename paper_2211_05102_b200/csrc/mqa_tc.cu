@@ -363,76 +363,129 @@ __device__ __noinline__ long long span_begin_nl(int i, int T, int G) { return sp
 //   M = max_s m_s;  out = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s
 // Every block that holds one of the sequence's `nparts` parts merges an equal slice of the [H, D] output
 // (block number `u` of them the u-th slice) once all parts have arrived, so the work after the last arrival is one
-// slice per block whatever the number of parts.  Parts are folded in block order with a running maximum and
-// each output element by exactly one thread: the result does not depend on timing.  The merge is bound by
-// round trips to L2, not by bytes, so a thread keeps the loads of several parts and output groups in flight.
-// All threads of the block call this; the blocks of one launch are co-resident (cooperative launch).
+// slice per block whatever the number of parts.  The merge is bound by round trips to L2, not by bytes:
+//   - a slice with at least as many float4 groups as threads: a thread folds all parts of EU groups, the loads
+//     of PB parts of each in flight together;
+//   - a smaller slice (many parts): the threads form `ngroups` groups, each folds a contiguous run of the parts
+//     for every float4 group of the slice, and the first group folds the groups' results from shared memory.
+// Parts and groups are folded in a fixed order, so the result does not depend on timing.
+// All threads of the block call this (it synchronises them); the blocks of one launch are co-resident.
+struct MergeState {
+    float M, Ls;
+    float4 acc;
+    __device__ __forceinline__ void init() { M = -INFINITY; Ls = 0.f; acc = make_float4(0.f, 0.f, 0.f, 0.f); }
+    __device__ __forceinline__ void fold(float ms, float ls, const float4& as) {
+        const float m_new = fmaxf(M, ms);
+        const float wa = (M == -INFINITY) ? 0.f : ex2_approx(M - m_new);
+        const float wb = (ms == -INFINITY) ? 0.f : ex2_approx(ms - m_new);
+        M = m_new;
+        Ls = fmaf(wa, Ls, wb * ls);
+        acc.x = fmaf(wa, acc.x, wb * as.x); acc.y = fmaf(wa, acc.y, wb * as.y);
+        acc.z = fmaf(wa, acc.z, wb * as.z); acc.w = fmaf(wa, acc.w, wb * as.w);
+    }
+};
+
 template <int D>
-__device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, long long P, int i_first, int first_slot, int u, int nparts, int nthreads)
+__device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, long long P, int i_first, int first_slot,
+                                         int u, int nparts, int nthreads, float* scratch)
 {
-    constexpr int PB = 4, EU = 2;
+    constexpr int PB = 4, EU = 3, PB1 = 6;
     const int H = p.H, Hp4 = round_up(H, 4);
     const int total = H * D / 4;                       // float4 groups of the output
     const int e_lo = total * u / nparts, e_hi = total * (u + 1) / nparts;   // total <= 4096, u < nparts <= 592
+    const int n_elem = e_hi - e_lo;
+    float4* const out4 = reinterpret_cast<float4*>(p.out + (size_t)b * H * D);
     // part s lives in the head slot of the s-th block that owns tiles of the sequence (the first part possibly in a tail slot)
     auto part_ptr = [&](int s) -> const float* {
         // T < G: one tile per block, and all of the arithmetic fits in 32 bits
         const int blk = (T >= G) ? i_first + s : (((int)P + s + 1) * G + T - 1) / T - 1;
         return ws_slot(p.workspace, p.B, H, D, s == 0 ? first_slot : 2 * blk);
     };
-    // EU output groups per thread and pass, PB parts each: EU*PB independent 16-byte loads in flight
-    for (int e0 = e_lo + (int)threadIdx.x; e0 < e_hi; e0 += EU * nthreads) {
-        float M[EU], Ls[EU];
-        float4 acc[EU];
+    const int tid = (int)threadIdx.x;
+    int ngroups = (n_elem > 0) ? nthreads / n_elem : 1;
+    if (ngroups > (nparts + PB1 - 1) / PB1) ngroups = (nparts + PB1 - 1) / PB1;   // no more groups than rounds to save
+    if (ngroups <= 1) {
+        for (int e0 = e_lo + tid; e0 < e_hi; e0 += EU * nthreads) {
+            MergeState st[EU];
 #pragma unroll
-        for (int k = 0; k < EU; ++k) { M[k] = -INFINITY; Ls[k] = 0.f; acc[k] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        for (int s0 = 0; s0 < nparts; s0 += PB) {
-            float ms[EU][PB], ls[EU][PB];
-            float4 as[EU][PB];
+            for (int k = 0; k < EU; ++k) st[k].init();
+            for (int s0 = 0; s0 < nparts; s0 += PB) {
+                float ms[EU][PB], ls[EU][PB];
+                float4 as[EU][PB];
 #pragma unroll
-            for (int i = 0; i < PB; ++i) {
-                if (s0 + i < nparts) {
-                    const float* sp = part_ptr(s0 + i);
+                for (int i = 0; i < PB; ++i) {
+                    if (s0 + i < nparts) {
+                        const float* sp = part_ptr(s0 + i);
 #pragma unroll
-                    for (int k = 0; k < EU; ++k) {
-                        const int e = e0 + k * nthreads;
-                        if (e < e_hi) {
-                            const int h = (e * 4) / D;
-                            ms[k][i] = __ldcg(sp + h);
-                            ls[k][i] = __ldcg(sp + Hp4 + h);
-                            as[k][i] = __ldcg(reinterpret_cast<const float4*>(sp + 2 * Hp4) + e);
+                        for (int k = 0; k < EU; ++k) {
+                            const int e = e0 + k * nthreads;
+                            if (e < e_hi) {
+                                const int h = (e * 4) / D;
+                                ms[k][i] = __ldcg(sp + h);
+                                ls[k][i] = __ldcg(sp + Hp4 + h);
+                                as[k][i] = __ldcg(reinterpret_cast<const float4*>(sp + 2 * Hp4) + e);
+                            }
                         }
                     }
                 }
+#pragma unroll
+                for (int i = 0; i < PB; ++i)
+                    if (s0 + i < nparts)
+#pragma unroll
+                        for (int k = 0; k < EU; ++k)
+                            if (e0 + k * nthreads < e_hi) st[k].fold(ms[k][i], ls[k][i], as[k][i]);
             }
 #pragma unroll
-            for (int i = 0; i < PB; ++i) {
-                if (s0 + i < nparts) {
-#pragma unroll
-                    for (int k = 0; k < EU; ++k) {
-                        if (e0 + k * nthreads < e_hi) {
-                            const float m_new = fmaxf(M[k], ms[k][i]);
-                            const float wa = (M[k] == -INFINITY) ? 0.f : ex2_approx(M[k] - m_new);
-                            const float wb = ex2_approx(ms[k][i] - m_new);
-                            M[k] = m_new;
-                            Ls[k] = fmaf(wa, Ls[k], wb * ls[k][i]);
-                            acc[k].x = fmaf(wa, acc[k].x, wb * as[k][i].x); acc[k].y = fmaf(wa, acc[k].y, wb * as[k][i].y);
-                            acc[k].z = fmaf(wa, acc[k].z, wb * as[k][i].z); acc[k].w = fmaf(wa, acc[k].w, wb * as[k][i].w);
-                        }
-                    }
+            for (int k = 0; k < EU; ++k) {
+                const int e = e0 + k * nthreads;
+                if (e < e_hi) {
+                    const float inv = __frcp_rn(st[k].Ls);
+                    out4[e] = make_float4(st[k].acc.x * inv, st[k].acc.y * inv, st[k].acc.z * inv, st[k].acc.w * inv);
                 }
             }
         }
+        return;
+    }
+    // many parts, small slice: group gi folds parts [s_lo, s_hi) of float4 group e_lo + ei
+    const int gi = tid / n_elem, ei = tid - gi * n_elem;
+    const int per = (nparts + ngroups - 1) / ngroups;
+    const int s_lo = gi * per, s_hi = min(nparts, s_lo + per);
+    const int e = e_lo + ei, h = (e * 4) / D;
+    MergeState st;
+    st.init();
+    if (gi < ngroups) {
+        for (int s0 = s_lo; s0 < s_hi; s0 += PB1) {
+            float ms[PB1], ls[PB1];
+            float4 as[PB1];
 #pragma unroll
-        for (int k = 0; k < EU; ++k) {
-            const int e = e0 + k * nthreads;
-            if (e < e_hi) {
-                const float inv = __frcp_rn(Ls[k]);
-                reinterpret_cast<float4*>(p.out + (size_t)b * H * D)[e] =
-                    make_float4(acc[k].x * inv, acc[k].y * inv, acc[k].z * inv, acc[k].w * inv);
+            for (int i = 0; i < PB1; ++i) {
+                if (s0 + i < s_hi) {
+                    const float* sp = part_ptr(s0 + i);
+                    ms[i] = __ldcg(sp + h);
+                    ls[i] = __ldcg(sp + Hp4 + h);
+                    as[i] = __ldcg(reinterpret_cast<const float4*>(sp + 2 * Hp4) + e);
+                }
             }
+#pragma unroll
+            for (int i = 0; i < PB1; ++i)
+                if (s0 + i < s_hi) st.fold(ms[i], ls[i], as[i]);
+        }
+        if (gi > 0) {
+            float* dst = scratch + ((size_t)(gi - 1) * n_elem + ei) * 8;
+            *reinterpret_cast<float4*>(dst) = st.acc;
+            dst[4] = st.M; dst[5] = st.Ls;
         }
     }
+    __syncthreads();
+    if (gi == 0) {
+        for (int g2 = 1; g2 < ngroups; ++g2) {
+            const float* src = scratch + ((size_t)(g2 - 1) * n_elem + ei) * 8;
+            st.fold(src[4], src[5], *reinterpret_cast<const float4*>(src));
+        }
+        const float inv = __frcp_rn(st.Ls);
+        out4[e] = make_float4(st.acc.x * inv, st.acc.y * inv, st.acc.z * inv, st.acc.w * inv);
+    }
+    __syncthreads();   // the scratch area may be reused by the next call
 }
 
 // Zero rows [first, 8192/D) of a staged V slot (D/64 boxes of [rows x 128 B]); called by a whole warp.  Rare
@@ -1124,12 +1177,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             if (tid == 0) PROF_TS(6);
             if (!__syncthreads_or(failed)) {
                 if (tid == 0) PROF_TS(8);
-                merge_slice<D>(p, T, G, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
-                if (ncut > 1) merge_slice<D>(p, T, G, cut1.b, cut1.P, cut1.i_first, cut1.first_slot, cut1.u, cut1.nparts, L::kThreads);
+                // the K/V ring is idle now: scratch for the merge (at most 32 bytes per thread)
+                float* scratch = reinterpret_cast<float*>(ring);
+                merge_slice<D>(p, T, G, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads, scratch);
+                if (ncut > 1)
+                    merge_slice<D>(p, T, G, cut1.b, cut1.P, cut1.i_first, cut1.first_slot, cut1.u, cut1.nparts, L::kThreads, scratch);
                 if (tid == 0) PROF_TS(9);
-#ifdef MQA_X_MERGE_TWICE
-                merge_slice<D>(p, T, G, cut0.b, cut0.P, cut0.i_first, cut0.first_slot, cut0.u, cut0.nparts, L::kThreads);
-#endif
                 __syncthreads();   // every thread of this block has read its parts
                 if (tid == 0) PROF_TS(10);
                 if (tid == 0) {
@@ -1260,9 +1313,6 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#ifdef MQA_X_COOP_ENV
-    if (const char* e3 = getenv("MQA_X_COOP")) cfg.numAttrs = atoi(e3);
-#endif
     return cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
 }
 
