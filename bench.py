@@ -294,7 +294,10 @@ def run_ours(args, w):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
         "data": "synthetic",
         "config": config_of(w, world, {
-            "plan": {"path": {1: "fma", 2: "tcgen05"}[plan.path], "num_ctas": plan.num_ctas, "tile_rows": plan.tile_rows},
+            "plan": {"path": {1: "fma", 2: "tcgen05"}[plan.path], "num_ctas": plan.num_ctas, "tile_rows": plan.tile_rows,
+                     "adaptive": bool(plan.adaptive),
+                     # blocks that took tiles in the last step (workspace header word 3, written by the kernel)
+                     "ctas_used": int(ws[:16].view(torch.int32)[3])},
             "l2": "inputs larger than L2" if kv_alloc >= 4 * l2_bytes else "L2 flushed between steps (flush untimed)",
             "ideal_kv_bytes_per_step": nbytes}),
         "pct_of_8000_GBps": 100.0 * value / world / NOMINAL_HBM_GBS,
