@@ -154,6 +154,29 @@ int mqa_append_decode(const void* q, const void* k_new, const void* v_new,
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Batch-sharded decode attention with the output already laid out for a heads-sharded consumer
+ * (Section 3.3: multiquery attention is sharded over the batch, at the price of an all-to-all that moves
+ * the per-token tensors between the heads-sharded and the batch-sharded layout; Figure 5).  This call is one
+ * rank's attention over its slice of the batch, fused with the all-to-all of the OUTPUT: instead of one
+ * [B,H,D] array, head h of local sequence b is stored to
+ *     out_dst[h / (H/n_dst)] + ((b_offset + b) * (H/n_dst) + h % (H/n_dst)) * D,
+ * i.e. into row b_offset + b of destination rank r's [B_total, H/n_dst, D] fp32 buffer.  The destinations are
+ * plain device pointers: this GPU's own memory, or peers' memory mapped into this process (peer access /
+ * symmetric memory over NVLink); the kernel reaches them with ordinary stores, never with TMA multicast.
+ *   out_dst   HOST array of n_dst device pointers (copied into the launch), each 16-byte aligned, each a
+ *             buffer of at least B_total * (H/n_dst) * D floats; rows outside [b_offset, b_offset + B) are
+ *             not touched
+ *   n_dst     1..16, a divisor of H;   b_offset >= 0, b_offset + B <= B_total
+ * The caller synchronises the ranks before the consumer reads (the stores are complete when the stream
+ * reaches the end of this call's kernel).  Tensor-core path only (D in {128, 256}): other shapes return
+ * MQA_ERR_UNSUPPORTED_SHAPE.  Everything else as mqa_decode.
+ */
+int mqa_decode_scatter(const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* lengths, float* const* out_dst, int n_dst, int b_offset, int B_total,
+                       int B, int H, int D, int Lmax, float scale,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Decode attention with KVH key/value heads per sequence (grouped-query attention; KVH == H is the
  * multihead attention the paper compares against in Section 4.2 and Table 1, KVH == 1 is mqa_decode).
  * Query head h uses key/value head h / (H/KVH).  The cache then holds KVH times the bytes, which is the

@@ -33,7 +33,7 @@ EXPORTS = [
     "mqa_status_string", "mqa_decode_workspace_bytes", "mqa_workspace_init", "mqa_decode_plan",
     "mqa_decode", "mqa_decode_with_plan", "mqa_decode_profiled", "mqa_check_status", "mqa_decode_host_scratch_bytes",
     "mqa_decode_host", "mqa_last_launch_count", "mqa_debug_schedule", "mqa_decode_static", "mqa_append_decode", "mqa_decode_grouped", "mqa_decode_grouped_workspace_bytes",
-    "mqa_uniform_ctas",
+    "mqa_uniform_ctas", "mqa_decode_scatter",
 ]
 
 
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.mqa_decode_grouped_workspace_bytes.restype = sz
         L.mqa_debug_schedule.argtypes = [vp, ci, ci, ci, ci, ci, vp, ci]; L.mqa_debug_schedule.restype = ci
         L.mqa_uniform_ctas.argtypes = [ci, ci, ci]; L.mqa_uniform_ctas.restype = ci
+        L.mqa_decode_scatter.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, sz, vp]
+        L.mqa_decode_scatter.restype = ci
         _lib = L
     return _lib
 
@@ -249,6 +251,30 @@ def mqa_decode_host(q, k_cache, v_cache, lengths, out, scale: float, scratch, st
 
 def mqa_last_launch_count() -> int:
     return int(lib().mqa_last_launch_count())
+
+
+def mqa_decode_scatter(q, k_cache, v_cache, lengths, out_dst, b_offset: int, scale: float, workspace, stream=None):
+    """One rank's batch-sharded decode attention with the output scattered by head group.
+
+    ``out_dst``: list of n_dst fp32 CUDA tensors [B_total, H/n_dst, D] (this GPU's or peers' memory), or a list of
+    (device pointer, B_total) pairs for memory that is not wrapped in a tensor.  Returns None."""
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.dim() == 3
+    B, H, D = q.shape
+    Lmax = k_cache.shape[1]
+    n_dst = len(out_dst)
+    ptrs, totals = [], []
+    for t in out_dst:
+        if isinstance(t, torch.Tensor):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.shape[1:] == (H // n_dst, D)
+            ptrs.append(t.data_ptr()); totals.append(t.shape[0])
+        else:
+            ptrs.append(int(t[0])); totals.append(int(t[1]))
+    assert len(set(totals)) == 1, "all destinations hold the same number of rows"
+    arr = (ctypes.c_void_p * n_dst)(*ptrs)
+    rc = lib().mqa_decode_scatter(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), lengths.data_ptr(),
+                                  arr, n_dst, int(b_offset), totals[0], B, H, D, Lmax, float(scale),
+                                  workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "mqa_decode_scatter")
 
 
 def mqa_uniform_ctas(B: int, tiles_per_sequence: int, num_ctas: int) -> int:

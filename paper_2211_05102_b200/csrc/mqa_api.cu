@@ -95,14 +95,29 @@ int mqa_decode_plan(int B, int H, int D, int Lmax, int requested_path, mqa_plan_
     return MQA_OK;
 }
 
+// Scattered output of mqa_decode_scatter (out is null then).
+struct ScatterArgs {
+    float* const* dst;   // host array of n_dst device pointers
+    int n_dst, b_offset, B_total;
+};
+
 static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* lengths, float* out,
                        int B, int H, int D, int Lmax, float scale,
                        const mqa_plan_t* plan,
                        void* workspace, size_t workspace_bytes, void* stream, void* event_after_split,
-                       int kv_groups = 1)
+                       int kv_groups = 1, const ScatterArgs* scatter = nullptr)
 {
-    if (!q || !k_cache || !v_cache || !lengths || !out || !workspace || !plan) return MQA_ERR_INVALID_ARG;
+    if (!q || !k_cache || !v_cache || !lengths || (!out && !scatter) || !workspace || !plan) return MQA_ERR_INVALID_ARG;
+    if (scatter) {
+        if (!scatter->dst || scatter->n_dst < 1 || scatter->n_dst > mqa::kMaxDst || scatter->b_offset < 0 ||
+            scatter->B_total < 1)
+            return MQA_ERR_INVALID_ARG;
+        if (H % scatter->n_dst != 0 || (long long)scatter->b_offset + B > scatter->B_total) return MQA_ERR_INVALID_ARG;
+        if (plan->path != MQA_PATH_TC) return MQA_ERR_UNSUPPORTED_SHAPE;   // only the tensor-core kernel scatters
+        for (int r = 0; r < scatter->n_dst; ++r)
+            if (!scatter->dst[r] || !aligned(scatter->dst[r], 16)) return scatter->dst[r] ? MQA_ERR_MISALIGNED : MQA_ERR_INVALID_ARG;
+    }
     if (B <= 0 || H <= 0 || D <= 0 || Lmax <= 0) return MQA_ERR_INVALID_ARG;
     if (!shape_ok(B, H, D, Lmax)) return MQA_ERR_UNSUPPORTED_SHAPE;
     if (!(scale == scale)) return MQA_ERR_INVALID_ARG;
@@ -111,7 +126,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     if (plan->tile_rows != ((plan->path == MQA_PATH_TC) ? 128 : 64)) return MQA_ERR_INVALID_ARG;
     if (plan->adaptive != 0 && plan->adaptive != 1) return MQA_ERR_INVALID_ARG;
     if (plan->path == MQA_PATH_TC && !mqa::tc_supported(H, D)) return MQA_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) ||
+    if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || (out && !aligned(out, 16)) ||
         !aligned(lengths, 4) || !aligned(workspace, 256))
         return MQA_ERR_MISALIGNED;
     if (workspace_bytes < mqa::workspace_bytes(B, H, D)) return MQA_ERR_WORKSPACE_TOO_SMALL;
@@ -130,6 +145,12 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.v = static_cast<const uint16_t*>(v_cache);
     p.lengths = mqa::LenView{lengths, kv_groups};
     p.out = out;
+    p.n_dst = 0; p.b_offset = 0;
+    for (int r = 0; r < mqa::kMaxDst; ++r) p.out_dst[r] = nullptr;
+    if (scatter) {
+        p.n_dst = scatter->n_dst; p.b_offset = scatter->b_offset;
+        for (int r = 0; r < scatter->n_dst; ++r) p.out_dst[r] = scatter->dst[r];
+    }
     p.B = B; p.H = H; p.D = D; p.Lmax = Lmax;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = tile_shift_of(plan->tile_rows);
@@ -191,6 +212,20 @@ int mqa_decode(const void* q, const void* k_cache, const void* v_cache,
     if (rc != MQA_OK) return rc;
     return mqa_decode_with_plan(q, k_cache, v_cache, lengths, out, B, H, D, Lmax, scale, &plan,
                                 workspace, workspace_bytes, stream);
+}
+
+int mqa_decode_scatter(const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* lengths, float* const* out_dst, int n_dst, int b_offset, int B_total,
+                       int B, int H, int D, int Lmax, float scale,
+                       void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (B <= 0 || H <= 0 || D <= 0 || Lmax <= 0) return MQA_ERR_INVALID_ARG;
+    mqa_plan_t plan;
+    const int rc = mqa_decode_plan(B, H, D, Lmax, MQA_PATH_TC, &plan);
+    if (rc != MQA_OK) return rc;
+    ScatterArgs sc{out_dst, n_dst, b_offset, B_total};
+    return decode_impl(q, k_cache, v_cache, lengths, nullptr, B, H, D, Lmax, scale, &plan,
+                       workspace, workspace_bytes, stream, nullptr, 1, &sc);
 }
 
 int mqa_append_decode(const void* q, const void* k_new, const void* v_new,

@@ -21,6 +21,7 @@ namespace mqa {
 constexpr int kHeaderBytes = 256;
 constexpr int kMaxCtas = 592;
 constexpr int kMaxHeads = 64;
+constexpr int kMaxDst = 16;               // destinations of a scattered output (ranks of one NVLink domain)
 
 // Workspace header words (int32).
 enum { kHdrStatus = 0, kHdrTotalTiles = 2, kHdrNumCtas = 3 };
@@ -63,7 +64,12 @@ struct Params {
     const uint16_t* k;        // [B,Lmax,D]
     const uint16_t* v;        // [B,Lmax,D]
     LenView lengths;          // [B / kv_groups] int32, viewed per (sequence, key/value head)
-    float* out;               // [B,H,D]
+    float* out;               // [B,H,D] (unused when the output is scattered)
+    // Scattered output (batch-sharded attention feeding a heads-sharded projection): head h of local sequence b
+    // goes to row (b_offset + b) of destination h / (H / n_dst), a [B_total, H / n_dst, D] buffer that may live
+    // in a peer GPU's memory.  n_dst = 0: plain output.
+    float* out_dst[kMaxDst];
+    int n_dst, b_offset;
     int B, H, D, Lmax;
     float scale_log2;         // scale * log2(e): logits are kept in the base-2 domain
     int tile_shift;           // log2(tile_rows)
@@ -72,6 +78,13 @@ struct Params {
     int lo_max_len;           // tensor-core path: sequences up to this length use hi+lo bf16 probabilities
     unsigned char* workspace;
 };
+
+// Address of output row (b, h): D contiguous floats.
+__device__ __forceinline__ float* out_row(const Params& p, int b, int h) {
+    if (p.n_dst == 0) return p.out + ((size_t)b * p.H + h) * p.D;
+    const int hpd = p.H / p.n_dst, r = h / hpd;
+    return p.out_dst[r] + ((size_t)(p.b_offset + b) * hpd + (h - r * hpd)) * p.D;
+}
 
 __host__ __device__ __forceinline__ int clamp_len(int len, int Lmax) { return len < 0 ? 0 : (len > Lmax ? Lmax : len); }
 

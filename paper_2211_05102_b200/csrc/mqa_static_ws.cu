@@ -98,6 +98,8 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     p.v = static_cast<const uint16_t*>(v_cache);
     p.lengths = mqa::LenView{lengths, 1};
     p.out = out;
+    p.n_dst = 0; p.b_offset = 0;
+    for (int r = 0; r < mqa::kMaxDst; ++r) p.out_dst[r] = nullptr;
     p.B = B; p.H = H; p.D = D; p.Lmax = Lmax;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.tile_shift = (plan.tile_rows == 128) ? 7 : 6;

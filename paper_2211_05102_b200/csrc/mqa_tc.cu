@@ -394,7 +394,8 @@ __device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, l
     const int total = H * D / 4;                       // float4 groups of the output
     const int e_lo = total * u / nparts, e_hi = total * (u + 1) / nparts;   // total <= 4096, u < nparts <= 592
     const int n_elem = e_hi - e_lo;
-    float4* const out4 = reinterpret_cast<float4*>(p.out + (size_t)b * H * D);
+    // float4 group e of sequence b: head e*4/D, offset e*4 - head*D within its row
+    auto out4 = [&](int e) -> float4* { const int h = (e * 4) / D; return reinterpret_cast<float4*>(out_row(p, b, h) + (e * 4 - h * D)); };
     // part s lives in the head slot of the s-th block that owns tiles of the sequence (the first part possibly in a tail slot)
     auto part_ptr = [&](int s) -> const float* {
         // T < G: one tile per block, and all of the arithmetic fits in 32 bits
@@ -440,7 +441,7 @@ __device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, l
                 const int e = e0 + k * nthreads;
                 if (e < e_hi) {
                     const float inv = __frcp_rn(st[k].Ls);
-                    out4[e] = make_float4(st[k].acc.x * inv, st[k].acc.y * inv, st[k].acc.z * inv, st[k].acc.w * inv);
+                    *out4(e) = make_float4(st[k].acc.x * inv, st[k].acc.y * inv, st[k].acc.z * inv, st[k].acc.w * inv);
                 }
             }
         }
@@ -483,7 +484,7 @@ __device__ __noinline__ void merge_slice(const Params& p, int T, int G, int b, l
             st.fold(src[4], src[5], *reinterpret_cast<const float4*>(src));
         }
         const float inv = __frcp_rn(st.Ls);
-        out4[e] = make_float4(st.acc.x * inv, st.acc.y * inv, st.acc.z * inv, st.acc.w * inv);
+        *out4(e) = make_float4(st.acc.x * inv, st.acc.y * inv, st.acc.z * inv, st.acc.w * inv);
     }
     __syncthreads();   // the scratch area may be reused by the next call
 }
@@ -589,8 +590,10 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     // Empty sequences own no tile: their output rows are zeroed here, round-robin over the blocks.
     for (int b = cta; b < p.B; b += (int)gridDim.x) {
         if (clamp_len(p.lengths[b], p.Lmax) == 0) {
-            float4* dst = reinterpret_cast<float4*>(p.out + (size_t)b * H * D);
-            for (int i = tid; i < H * D / 4; i += L::kThreads) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = tid; i < H * D / 4; i += L::kThreads) {
+                const int h = (i * 4) / D;
+                *reinterpret_cast<float4*>(out_row(p, b, h) + (i * 4 - h * D)) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
     }
 
@@ -939,16 +942,31 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                     float inv[HPT];
 #pragma unroll
                     for (int i = 0; i < HPT; ++i) inv[i] = __frcp_rn(misc.lsum[set][hb + i]);
+                    if (p.n_dst == 0) {
 #pragma unroll
-                    for (int j = 0; j < NACC; ++j) {
-                        float* dst = p.out + ((size_t)b * H + hb) * D + j * 128 + row;
+                        for (int j = 0; j < NACC; ++j) {
+                            float* dst = p.out + ((size_t)b * H + hb) * D + j * 128 + row;
 #pragma unroll
-                        for (int i = 0; i < HPT; ++i)
+                            for (int i = 0; i < HPT; ++i)
 #ifdef MQA_X_NOSTORE
-                            if (hb + i < H && inv[i] == 12345.f) dst[(size_t)i * D] = o[j][i] * inv[i];
+                                if (hb + i < H && inv[i] == 12345.f) dst[(size_t)i * D] = o[j][i] * inv[i];
 #else
-                            if (hb + i < H) __stcs(dst + (size_t)i * D, o[j][i] * inv[i]);
+                                if (hb + i < H) __stcs(dst + (size_t)i * D, o[j][i] * inv[i]);
 #endif
+                        }
+                    } else {
+                        // scattered output: consecutive heads walk through the destinations (H / n_dst heads each)
+                        const int hpd = H / p.n_dst;
+                        int r = hb / hpd, hh = hb - r * hpd;
+#pragma unroll
+                        for (int i = 0; i < HPT; ++i) {
+                            if (hb + i < H) {
+                                float* dst = p.out_dst[r] + ((size_t)(p.b_offset + b) * hpd + hh) * D + row;
+#pragma unroll
+                                for (int j = 0; j < NACC; ++j) __stcs(dst + j * 128, o[j][i] * inv[i]);
+                            }
+                            if (++hh == hpd) { hh = 0; ++r; }
+                        }
                     }
                 } else {
 #pragma unroll
