@@ -202,3 +202,35 @@ def test_cuda_graph_capture_and_replay():
     assert binding.mqa_check_status(ws) == binding.MQA_OK
     expect = ref.mqa_decode_ref(q2, k, v, ln, 1 / 16)
     assert_close(out.cpu(), expect, "graph replay with new q")
+
+
+def test_random_shapes_and_block_counts():
+    """Seeded sweep over shapes, length mixes and block counts (pinned and adaptive): every case against the
+    oracle.  Exercises cut sequences with 2..40 parts, blocks without tiles, empty sequences, one-row
+    sequences and uniform batches in one run."""
+    rng = np.random.default_rng(20221105)
+    worst = 0.0
+    for case in range(36):
+        D = int(rng.choice([128, 256]))
+        H = int(rng.choice([1, 3, 8, 16, 17, 32, 40, 48, 64]))
+        B = int(rng.integers(1, 41))
+        Lmax = int(rng.choice([130, 700, 2100, 5200]))
+        kind = case % 4
+        if kind == 0:
+            lengths = [int(x) for x in rng.integers(0, Lmax + 1, size=B)]
+        elif kind == 1:
+            lengths = [Lmax - int(x) for x in rng.integers(0, 100, size=B)]          # equal tile counts, mostly
+        elif kind == 2:
+            lengths = [int(rng.choice([0, 1, 127, 128, 129, Lmax])) for _ in range(B)]
+        else:
+            lengths = [Lmax] * B
+        q, k, v, ln = make_custom(B, H, D, Lmax, seed=3000 + case, lengths=lengths)
+        k, v = poison_padding(k, v, ln, 0x7FC0)
+        scale = 1.0 / math.sqrt(D)
+        expect = ref.mqa_decode_ref(q, k, v, ln, scale)
+        base = binding.mqa_decode_plan(B, H, D, Lmax, binding.MQA_PATH_TC)
+        pinned = binding.Plan(base.path, int(rng.integers(1, 149)), base.tile_rows)
+        for plan in (base, pinned):
+            got = run_gpu(q, k, v, ln, scale, plan=plan)
+            worst = max(worst, assert_close(got, expect, f"case {case}: B={B} H={H} D={D} Lmax={Lmax} kind={kind} {plan}"))
+    print(f"random sweep: max err/tol = {worst:.3f}")
