@@ -117,7 +117,7 @@ __host__ __device__ inline int uniform_ctas(int B, int nt, int G)
 {
     constexpr float kPerSmTileNs = 2330.f, kSmsToSaturate = 123.f, kCutSavingNs = 7000.f;
     const long long T = (long long)B * nt;
-    if (nt <= 0 || T <= G) return G;
+    if (nt <= 1 || T <= G) return G;                  // one tile per sequence: every cut is on a boundary already
     auto stream_ns = [&](int g) { return (float)T * kPerSmTileNs / (g < kSmsToSaturate ? (float)g : kSmsToSaturate); };
     int cand = 0;
     if (B >= G) {
