@@ -234,3 +234,36 @@ def test_random_shapes_and_block_counts():
             got = run_gpu(q, k, v, ln, scale, plan=plan)
             worst = max(worst, assert_close(got, expect, f"case {case}: B={B} H={H} D={D} Lmax={Lmax} kind={kind} {plan}"))
     print(f"random sweep: max err/tol = {worst:.3f}")
+
+
+@pytest.mark.parametrize("pin", [None, 148, 37])
+def test_repeated_launches_are_bit_identical(pin):
+    """Many back-to-back steps on a batch whose sequences are cut into 2..40 parts (publisher, arrival counters
+    that wrap back to zero, sliced merge): every step must reproduce the first one bit for bit, and the first
+    one must match the oracle.  A merge that read a part too early, or a counter that did not return to zero,
+    shows up here."""
+    B, H, D, Lmax = 12, 48, 256, 5200
+    lengths = [5200, 130, 0, 4100, 2600, 1, 900, 5199, 3333, 128, 777, 2048]
+    dev = torch.device("cuda:0")
+    q, k, v, ln = make_custom(B, H, D, Lmax, seed=911, lengths=lengths)
+    qd, kd, vd, ld = q.to(dev), k.to(dev), v.to(dev), ln.to(dev)
+    out = torch.empty((B, H, D), dtype=torch.float32, device=dev)
+    ws = binding.alloc_workspace(B, H, D, Lmax)
+    plan = binding.mqa_decode_plan(B, H, D, Lmax, binding.MQA_PATH_TC)
+    if pin is not None:
+        plan = binding.Plan(plan.path, pin, plan.tile_rows)
+    binding.mqa_decode(qd, kd, vd, ld, out, 1 / 16, ws, plan=plan)
+    torch.cuda.synchronize()
+    first = out.clone()
+    assert_close(first.cpu(), ref.mqa_decode_ref(q, k, v, ln, 1 / 16), f"first step, pin={pin}")
+    for it in range(400):
+        if it % 50 == 0:
+            out.fill_(float("nan"))
+        binding.mqa_decode(qd, kd, vd, ld, out, 1 / 16, ws, plan=plan)
+        if it % 50 == 49:
+            torch.cuda.synchronize()
+            assert torch.equal(out, first), f"step {it} differs"
+    assert binding.mqa_check_status(ws) == binding.MQA_OK
+    # the arrival counters are back at zero
+    off = 256 + (B * 8 + 255) // 256 * 256
+    assert int(ws[off:off + 4 * B].view(torch.int32).abs().sum()) == 0
