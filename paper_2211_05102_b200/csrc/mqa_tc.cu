@@ -558,18 +558,31 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
 #endif
     const int cta = blockIdx.x, H = p.H;
 
-    if (tid == 0) {
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
-        for (int i = 0; i < 2; ++i) {
+    // Barrier set-up is spread over the first threads (one thread doing all ~45 inits in a row is on every
+    // launch's critical path); the tensor maps are fetched ahead of the first loads.
+    {
+        constexpr uint32_t W = L::kSoftmaxThreads / 32;
+        if (tid < kMaxSlots) {
+            mbar_init(&bars.full[tid], 1); mbar_init(&bars.empty[tid], 1);
+        } else if (tid < kMaxSlots + 4) {
+            const int i = tid - kMaxSlots;
+            mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], W);
+        } else if (tid < kMaxSlots + 6) {
+            const int i = tid - kMaxSlots - 4;
             mbar_init(&bars.q_full[i], 1); mbar_init(&bars.q_empty[i], 1);
+            mbar_init(&bars.p_full[i], W); mbar_init(&bars.p_empty[i], 1);
+            mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], W);
+            mbar_init(&bars.pub[i], W);
+        } else if (tid == kMaxSlots + 6) {
+            misc.abort_flag = 0;
+            asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
         }
-        for (int i = 0; i < 4; ++i) { mbar_init(&bars.s_full[i], 1); mbar_init(&bars.s_empty[i], L::kSoftmaxThreads / 32); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bars.p_full[i], L::kSoftmaxThreads / 32); mbar_init(&bars.p_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], L::kSoftmaxThreads / 32); }
-        for (int i = 0; i < 2; ++i) mbar_init(&bars.pub[i], L::kSoftmaxThreads / 32);
-        misc.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_proxy_async();
+        if (tid < kMaxSlots + 6) {
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            fence_proxy_async();
+        }
     }
     if (warp == 1) {   // tensor-memory allocation (one warp owns it for the whole kernel)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc.tmem_base)), "r"(kTmemCols) : "memory");
