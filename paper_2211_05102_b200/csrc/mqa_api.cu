@@ -156,6 +156,7 @@ static int decode_impl(const void* q, const void* k_cache, const void* v_cache,
     p.tile_shift = tile_shift_of(plan->tile_rows);
     p.num_ctas = plan->num_ctas;
     p.adaptive = (plan->path == MQA_PATH_TC) ? plan->adaptive : 0;
+    p.cluster = 1;
     // The tensor-core kernel's blocks wait for one another (merge of cut sequences), so all of them must be
     // resident at once: one block per SM at most.
     if (plan->path == MQA_PATH_TC && p.num_ctas > sm_count_or_default()) p.num_ctas = sm_count_or_default();

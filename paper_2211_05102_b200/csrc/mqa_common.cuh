@@ -24,7 +24,7 @@ constexpr int kMaxHeads = 64;
 constexpr int kMaxDst = 16;               // destinations of a scattered output (ranks of one NVLink domain)
 
 // Workspace header words (int32).
-enum { kHdrStatus = 0, kHdrTotalTiles = 2, kHdrNumCtas = 3 };
+enum { kHdrStatus = 0, kHdrTotalTiles = 2, kHdrNumCtas = 3, kHdrPairMode = 4 };
 
 // Per-sequence record written by the block that owns the sequence's first tile.
 struct SeqInfo {
@@ -75,6 +75,7 @@ struct Params {
     int tile_shift;           // log2(tile_rows)
     int num_ctas;             // G (an upper bound when `adaptive` is set)
     int adaptive;             // tensor-core path: the kernel may run a uniform batch on fewer blocks (uniform_ctas)
+    int cluster;              // thread blocks per cluster of this launch (1, or 2: pairs may merge through shared memory)
     int lo_max_len;           // tensor-core path: sequences up to this length use hi+lo bf16 probabilities
     unsigned char* workspace;
 };
@@ -142,6 +143,7 @@ struct SchedShared {
     int p0;         // global index of that sequence's first tile
     long long g0, g1;   // this block's run of tiles [g0, g1)
     int G;              // blocks that share the tiles (the launch's block count unless the plan is adaptive)
+    int pair;           // uniform batch run on exactly two blocks per sequence (halves), see uniform_ctas
 };
 
 // Block-wide: total tile count T, and (b0, p0) for the tile `g0 = span_begin(cta)`.
@@ -186,7 +188,7 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
     __syncthreads();
     const int T = sh.total;
     if (uniform) G = uniform_ctas(B, nt_first, G);    // identical in every thread of every block
-    if (tid == 0) sh.G = G;
+    if (tid == 0) { sh.G = G; sh.pair = (uniform && G == 2 * B && (nt_first & 1) == 0) ? 1 : 0; }
     int prefix = sh.warp_sums[warp] + incl - local;   // tiles before this thread's first sequence
     if (T > 0 && cta < G) {
         const long long g0 = span_begin(cta, T, G);

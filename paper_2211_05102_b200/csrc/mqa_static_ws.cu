@@ -105,6 +105,7 @@ extern "C" int mqa_decode_static(const void* q, const void* k_cache, const void*
     p.tile_shift = (plan.tile_rows == 128) ? 7 : 6;
     p.num_ctas = plan.num_ctas;
     p.adaptive = (plan.path == MQA_PATH_TC) ? plan.adaptive : 0;
+    p.cluster = 1;
     p.lo_max_len = 0x7fffffff;
     p.workspace = ws;
     cudaError_t e = (plan.path == MQA_PATH_TC) ? mqa::launch_tc(p, st) : mqa::launch_fma(p, st);

@@ -64,6 +64,7 @@ struct Barriers {
     unsigned long long p_full[2], p_empty[2];
     unsigned long long o_full[2], o_empty[2];
     unsigned long long pub[2];     // softmax warps -> publisher warp: the partial result in slot 2*cta + j is stored
+    unsigned long long xbar;       // pair mode: the partner block's softmax warps have delivered their half (cluster scope)
 };
 
 struct Misc {
@@ -78,6 +79,7 @@ struct Misc {
     __align__(16) float m[kMaxHeads];      // reference maximum per head of the current segment (base-2 domain)
     __align__(16) float alpha[kMaxHeads];  // rescale factors
     __align__(16) float lsum[2][kMaxHeads]; // row sums of a finished segment, by segment parity, until its epilogue has run
+    float xm[kMaxHeads];           // pair mode: the partner's reference maxima (its row sums arrive in lsum[1])
 };
 
 // Optional cycle accounting (compile with -DMQA_TC_PROFILE): block 0 adds the cycles each role
@@ -179,6 +181,38 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
 }
 
 // Arrive on an mbarrier once every MMA issued so far by this thread has completed.
+// ---- thread-block cluster helpers (pair mode: two blocks of one sequence exchange halves through shared memory)
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {   // same offset in another block's shared memory
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t raddr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(raddr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t raddr) {   // release at cluster scope: the stores above are visible to the waiter
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(raddr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(void* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __noinline__ bool mbar_wait_cluster(void* bar, uint32_t parity, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((spins & 63u) == 0u && (clock64() - t0 > kWaitLimitCycles || *abort_flag)) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void cluster_sync_all() {   // every thread of every block of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void umma_commit(void* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -532,7 +566,7 @@ struct TcLayout {
 
 template <int D, int HP>
 __global__ void __launch_bounds__(TcLayout<D, HP>::kThreads, 1)
-mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+mqa_tc_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, const int nslots)
 {
     using L = TcLayout<D, HP>;
@@ -574,12 +608,13 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             mbar_init(&bars.o_full[i], 1); mbar_init(&bars.o_empty[i], W);
             mbar_init(&bars.pub[i], W);
         } else if (tid == kMaxSlots + 6) {
+            mbar_init(&bars.xbar, W);
             misc.abort_flag = 0;
             asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
             asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
             asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
         }
-        if (tid < kMaxSlots + 6) {
+        if (tid <= kMaxSlots + 6) {
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             fence_proxy_async();
         }
@@ -592,6 +627,12 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     const int T = schedule_prologue<L::kThreads>(p.lengths, p.B, p.Lmax, kTileShift, p.num_ctas, cta, misc.sched,
                                                  p.adaptive != 0);   // has __syncthreads
     const int G = misc.sched.G;   // blocks that share the tiles (fewer than launched for some uniform batches)
+    // Pair mode: a uniform batch on exactly two blocks per sequence, launched as clusters of two (consecutive block
+    // numbers = the two halves of one sequence): the halves are merged through distributed shared memory instead of
+    // global memory.  The partner's barrier must exist before anything is sent to it.
+    if (p.cluster > 1) cluster_sync_all();
+    const bool pair = p.cluster == 2 && NACC == 2 && misc.sched.pair != 0;
+    if (cta == 0 && tid == 0) ws_header(p.workspace)[kHdrPairMode] = pair ? 1 : 0;
     tc_fence_after();
     const uint32_t tmem = misc.tmem_base;
     if (cta == 0 && tid == 0) {
@@ -879,7 +920,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
             // its parts have arrived).  Keeping the fence and the atomic here keeps them off the softmax warps.
             SegmentWalker w;
             w.init_span(p.lengths, p.B, p.Lmax, kTileShift, misc.sched.g0, misc.sched.g1, misc.sched.b0, misc.sched.p0);
-            while (!w.done()) {
+            while (!pair && !w.done()) {
                 if (!w.seg_is_whole()) {
                     if (!mbar_wait(&bars.pub[w.seg_slot(cta) & 1], 0, abort_flag)) break;
                     if (lane == 0) {
@@ -939,7 +980,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 PROF_BEGIN();
                 float* slot_ptr = whole ? nullptr : ws_slot(p.workspace, p.B, H, D, pend.slot_id);
                 const int Hp4 = round_up(H, 4);
-                if (!whole && row < HPT && hmine < H) {
+                if (!whole && !pair && row < HPT && hmine < H) {
                     slot_ptr[hmine] = pend.m_mine;
                     slot_ptr[Hp4 + hmine] = misc.lsum[set][hmine];
                 }
@@ -951,6 +992,56 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars.o_empty[set]);   // the accumulators are in registers now
                 TRACE(2, 42, pend.seg);
+                if (pair) {
+                    // This block holds one half of the sequence's tiles, its cluster partner the other.  Block u
+                    // finishes output columns [128u, 128u+128): it sends the other 128 columns of its accumulator,
+                    // and its reference maxima and row sums, into the partner's shared memory (the idle second q
+                    // buffer, xm, lsum[1]), then folds what the partner sent into the half it keeps.
+                    const uint32_t u = cluster_ctarank(), peer = u ^ 1u;
+                    float* xbuf = reinterpret_cast<float*>(q_buf + L::kQBytes);          // [head][128 columns]
+                    const uint32_t r_x = map_to_cta(smem_u32(xbuf), peer);
+                    float keep[HPT], send[HPT];                  // (plain copies under a uniform branch keep o[][] in registers)
+                    if (u == 0) {
+#pragma unroll
+                        for (int i = 0; i < HPT; ++i) { keep[i] = o[0][i]; send[i] = o[1][i]; }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < HPT; ++i) { keep[i] = o[1][i]; send[i] = o[0][i]; }
+                    }
+                    if (row < HPT && hmine < H) {
+                        st_cluster_f32(map_to_cta(smem_u32(&misc.xm[hmine]), peer), pend.m_mine);
+                        st_cluster_f32(map_to_cta(smem_u32(&misc.lsum[1][hmine]), peer), misc.lsum[set][hmine]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < HPT; ++i)
+                        if (hb + i < H) st_cluster_f32(r_x + 4u * (uint32_t)((hb + i) * 128 + row), send[i]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars.xbar), peer));
+                    {   // the partner's half (bounded wait; the first warp of the group polls, the rest follow it)
+                        bool failed = false;
+                        if (wq == 0 && !mbar_try_wait_cluster(&bars.xbar, 0)) failed = !mbar_wait_cluster(&bars.xbar, 0, abort_flag);
+                        if (softmax_bar_or(failed, NSM)) return false;
+                    }
+#pragma unroll
+                    for (int i = 0; i < HPT; ++i) {
+                        const int h = hb + i;
+                        if (h < H) {
+                            // part 0 is the first half of the rows: fold in that order on both sides
+                            const float m_own = misc.m[h], l_own = misc.lsum[set][h], o_own = keep[i];
+                            const float m_oth = misc.xm[h], l_oth = misc.lsum[1][h], o_oth = xbuf[h * 128 + row];
+                            const float m0 = u == 0 ? m_own : m_oth, m1 = u == 0 ? m_oth : m_own;
+                            const float l0 = u == 0 ? l_own : l_oth, l1 = u == 0 ? l_oth : l_own;
+                            const float a0 = u == 0 ? o_own : o_oth, a1 = u == 0 ? o_oth : o_own;
+                            const float M = fmaxf(m0, m1);
+                            const float w0 = ex2_approx(m0 - M), w1 = ex2_approx(m1 - M);
+                            const float num = fmaf(w0, a0, w1 * a1), den = fmaf(w0, l0, w1 * l1);
+                            __stcs(out_row(p, b, h) + 128 * (int)u + row, num * __frcp_rn(den));
+                        }
+                    }
+                    TRACE(2, 43, pend.seg);
+                    PROF_END(kProfSmEpilogue);
+                    return true;
+                }
                 if (whole) {
                     float inv[HPT];
 #pragma unroll
@@ -1173,7 +1264,7 @@ mqa_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_q, const _
     // a bounded wait.  The counter runs on to 2*nparts as the blocks leave; the last one out zeroes it for the
     // next call.
 #ifndef MQA_X_SKIP_MERGE
-    if (!misc.abort_flag && N > 0) {
+    if (!misc.abort_flag && N > 0 && !pair) {
         struct Cut { int b, i_first, first_slot, u, nparts; long long P; };
         Cut cut0 = {}, cut1 = {};
         int ncut = 0;
@@ -1339,11 +1430,37 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
     cfg.blockDim = dim3((unsigned)L::kThreads);
     cfg.dynamicSmemBytes = (size_t)L::smem_bytes(nslots);
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // Clusters of two when the split-count heuristic would cut every sequence of a full-length uniform batch into
+    // two halves: consecutive blocks then hold the halves of one sequence and merge them through distributed
+    // shared memory (the kernel checks on the device that the batch really is uniform; otherwise the pairs are
+    // simply not used).  The host sees only Lmax, so the prediction assumes every sequence fills its cache.
+    p.cluster = 1;
+    if (D == 256 && p.adaptive && (p.num_ctas % 2) == 0 &&
+        uniform_ctas(p.B, (p.Lmax + kTileRows - 1) / kTileRows, p.num_ctas) == 2 * p.B) {
+        static int s_pairs_fit[kMaxDevices] = {};   // 0 unknown, 1 yes, -1 no
+        if (s_pairs_fit[dev] == 0) {
+            cudaLaunchConfig_t probe = cfg;
+            cudaLaunchAttribute pa[1];
+            pa[0].id = cudaLaunchAttributeClusterDimension;
+            pa[0].val.clusterDim.x = 2; pa[0].val.clusterDim.y = 1; pa[0].val.clusterDim.z = 1;
+            probe.attrs = pa; probe.numAttrs = 1;
+            int nclusters = 0;
+            const cudaError_t qe = cudaOccupancyMaxActiveClusters(&nclusters, mqa_tc_kernel<D, HP>, &probe);
+            if (qe != cudaSuccess) cudaGetLastError();
+            s_pairs_fit[dev] = (qe == cudaSuccess && 2 * nclusters >= p.num_ctas) ? 1 : -1;
+        }
+        if (s_pairs_fit[dev] == 1) {
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+            p.cluster = 2;
+        }
+    }
     return cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
 }
 

@@ -267,3 +267,31 @@ def test_repeated_launches_are_bit_identical(pin):
     # the arrival counters are back at zero
     off = 256 + (B * 8 + 255) // 256 * 256
     assert int(ws[off:off + 4 * B].view(torch.int32).abs().sum()) == 0
+
+
+@pytest.mark.parametrize("B,H,L", [(64, 32, 2048), (70, 48, 512), (37, 64, 1024), (74, 16, 300), (64, 48, 4096)])
+def test_pair_mode_merges_halves_through_cluster_shared_memory(B, H, L):
+    """Uniform batches that the heuristic runs on exactly two blocks per sequence: the launch uses clusters of
+    two and the halves are merged through distributed shared memory (workspace header word 4 says so).
+    Unequal lengths inside the same tile count, padding poisoned with NaN."""
+    D, Lmax = 256, L
+    lengths = [L - (i % 5) for i in range(B)]
+    q, k, v, ln = make_custom(B, H, D, Lmax, seed=5150 + B, lengths=lengths)
+    k, v = poison_padding(k, v, ln, 0x7FC0)
+    expect = ref.mqa_decode_ref(q, k, v, ln, 1.0 / math.sqrt(D))
+    ws = binding.alloc_workspace(B, H, D, Lmax)
+    got = run_gpu(q, k, v, ln, 1.0 / math.sqrt(D), workspace=ws)
+    assert_close(got, expect, f"pair mode B={B} H={H} L={L}")
+    hdr = ws[:32].view(torch.int32)
+    plan = binding.mqa_decode_plan(B, H, D, Lmax, binding.MQA_PATH_TC)
+    if binding.mqa_uniform_ctas(B, (L + 127) // 128, plan.num_ctas) == 2 * B and plan.num_ctas % 2 == 0:
+        assert int(hdr[4]) == 1, "expected the pair path"
+        assert int(hdr[3]) == 2 * B
+    again = run_gpu(q, k, v, ln, 1.0 / math.sqrt(D), workspace=ws)
+    assert torch.equal(got, again)
+    # a ragged batch of the same shape falls back to the global-memory merge in the same cluster launch
+    lengths2 = [max(1, L - 137 * i) for i in range(B)]
+    q2, k2, v2, ln2 = make_custom(B, H, D, Lmax, seed=5151 + B, lengths=lengths2)
+    assert_close(run_gpu(q2, k2, v2, ln2, 1.0 / math.sqrt(D), workspace=ws),
+                 ref.mqa_decode_ref(q2, k2, v2, ln2, 1.0 / math.sqrt(D)), "ragged under a cluster launch")
+    assert int(ws[:32].view(torch.int32)[4]) == 0
