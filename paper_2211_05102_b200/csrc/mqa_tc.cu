@@ -984,6 +984,65 @@ mqa_tc_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensor
                     slot_ptr[hmine] = pend.m_mine;
                     slot_ptr[Hp4 + hmine] = misc.lsum[set][hmine];
                 }
+                if (pair) {
+                    // This block holds one half of the sequence's tiles, its cluster partner the other.  Block u
+                    // finishes output columns [128u, 128u+128): it sends the other 128 columns of its accumulator,
+                    // and its reference maxima and row sums, into the partner's shared memory (the idle second q
+                    // buffer, xm, lsum[1]), then folds what the partner sent into the half it keeps.
+                    // The accumulator is read from tensor memory eight heads at a time in rolled loops: this code
+                    // runs once per launch, so its instruction fetches, not its instruction count, set its cost.
+                    const uint32_t u = cluster_ctarank(), peer = u ^ 1u;
+                    float* xbuf = reinterpret_cast<float*>(q_buf + L::kQBytes);          // [head][128 columns]
+                    const uint32_t r_x = map_to_cta(smem_u32(xbuf), peer);
+                    const uint32_t t_send = lane_base + kOCol + (uint32_t)(set * 128 + (int)peer * 64 + hb);
+                    const uint32_t t_keep = lane_base + kOCol + (uint32_t)(set * 128 + (int)u * 64 + hb);
+                    if (row < HPT && hmine < H) {
+                        st_cluster_f32(map_to_cta(smem_u32(&misc.xm[hmine]), peer), pend.m_mine);
+                        st_cluster_f32(map_to_cta(smem_u32(&misc.lsum[1][hmine]), peer), misc.lsum[set][hmine]);
+                    }
+#pragma unroll 1
+                    for (int c8 = 0; c8 < HPT; c8 += 8) {
+                        float v[8];
+                        tmem_ld<8>(t_send + (uint32_t)c8, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (hb + c8 + i < H) st_cluster_f32(r_x + 4u * (uint32_t)((hb + c8 + i) * 128 + row), v[i]);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars.xbar), peer));
+                    {   // the partner's half (bounded wait; the first warp of the group polls, the rest follow it)
+                        bool failed = false;
+                        if (wq == 0 && !mbar_try_wait_cluster(&bars.xbar, 0)) failed = !mbar_wait_cluster(&bars.xbar, 0, abort_flag);
+                        if (softmax_bar_or(failed, NSM)) return false;
+                    }
+#pragma unroll 1
+                    for (int c8 = 0; c8 < HPT; c8 += 8) {
+                        float v[8];
+                        tmem_ld<8>(t_keep + (uint32_t)c8, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int h = hb + c8 + i;
+                            if (h < H) {
+                                // part 0 is the first half of the rows: fold in that order on both sides
+                                const float m_own = misc.m[h], l_own = misc.lsum[set][h], o_own = v[i];
+                                const float m_oth = misc.xm[h], l_oth = misc.lsum[1][h], o_oth = xbuf[h * 128 + row];
+                                const float m0 = u == 0 ? m_own : m_oth, m1 = u == 0 ? m_oth : m_own;
+                                const float l0 = u == 0 ? l_own : l_oth, l1 = u == 0 ? l_oth : l_own;
+                                const float a0 = u == 0 ? o_own : o_oth, a1 = u == 0 ? o_oth : o_own;
+                                const float M = fmaxf(m0, m1);
+                                const float w0 = ex2_approx(m0 - M), w1 = ex2_approx(m1 - M);
+                                const float num = fmaf(w0, a0, w1 * a1), den = fmaf(w0, l0, w1 * l1);
+                                __stcs(out_row(p, b, h) + 128 * (int)u + row, num * __frcp_rn(den));
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    TRACE(2, 43, pend.seg);
+                    PROF_END(kProfSmEpilogue);
+                    return true;
+                }
                 float o[NACC][HPT];
 #pragma unroll
                 for (int j = 0; j < NACC; ++j) tmem_ld<HPT>(lane_base + kOCol + (uint32_t)(set * 128 + j * 64 + hb), o[j]);
@@ -992,56 +1051,6 @@ mqa_tc_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensor
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars.o_empty[set]);   // the accumulators are in registers now
                 TRACE(2, 42, pend.seg);
-                if (pair) {
-                    // This block holds one half of the sequence's tiles, its cluster partner the other.  Block u
-                    // finishes output columns [128u, 128u+128): it sends the other 128 columns of its accumulator,
-                    // and its reference maxima and row sums, into the partner's shared memory (the idle second q
-                    // buffer, xm, lsum[1]), then folds what the partner sent into the half it keeps.
-                    const uint32_t u = cluster_ctarank(), peer = u ^ 1u;
-                    float* xbuf = reinterpret_cast<float*>(q_buf + L::kQBytes);          // [head][128 columns]
-                    const uint32_t r_x = map_to_cta(smem_u32(xbuf), peer);
-                    float keep[HPT], send[HPT];                  // (plain copies under a uniform branch keep o[][] in registers)
-                    if (u == 0) {
-#pragma unroll
-                        for (int i = 0; i < HPT; ++i) { keep[i] = o[0][i]; send[i] = o[1][i]; }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < HPT; ++i) { keep[i] = o[1][i]; send[i] = o[0][i]; }
-                    }
-                    if (row < HPT && hmine < H) {
-                        st_cluster_f32(map_to_cta(smem_u32(&misc.xm[hmine]), peer), pend.m_mine);
-                        st_cluster_f32(map_to_cta(smem_u32(&misc.lsum[1][hmine]), peer), misc.lsum[set][hmine]);
-                    }
-#pragma unroll
-                    for (int i = 0; i < HPT; ++i)
-                        if (hb + i < H) st_cluster_f32(r_x + 4u * (uint32_t)((hb + i) * 128 + row), send[i]);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars.xbar), peer));
-                    {   // the partner's half (bounded wait; the first warp of the group polls, the rest follow it)
-                        bool failed = false;
-                        if (wq == 0 && !mbar_try_wait_cluster(&bars.xbar, 0)) failed = !mbar_wait_cluster(&bars.xbar, 0, abort_flag);
-                        if (softmax_bar_or(failed, NSM)) return false;
-                    }
-#pragma unroll
-                    for (int i = 0; i < HPT; ++i) {
-                        const int h = hb + i;
-                        if (h < H) {
-                            // part 0 is the first half of the rows: fold in that order on both sides
-                            const float m_own = misc.m[h], l_own = misc.lsum[set][h], o_own = keep[i];
-                            const float m_oth = misc.xm[h], l_oth = misc.lsum[1][h], o_oth = xbuf[h * 128 + row];
-                            const float m0 = u == 0 ? m_own : m_oth, m1 = u == 0 ? m_oth : m_own;
-                            const float l0 = u == 0 ? l_own : l_oth, l1 = u == 0 ? l_oth : l_own;
-                            const float a0 = u == 0 ? o_own : o_oth, a1 = u == 0 ? o_oth : o_own;
-                            const float M = fmaxf(m0, m1);
-                            const float w0 = ex2_approx(m0 - M), w1 = ex2_approx(m1 - M);
-                            const float num = fmaf(w0, a0, w1 * a1), den = fmaf(w0, l0, w1 * l1);
-                            __stcs(out_row(p, b, h) + 128 * (int)u + row, num * __frcp_rn(den));
-                        }
-                    }
-                    TRACE(2, 43, pend.seg);
-                    PROF_END(kProfSmEpilogue);
-                    return true;
-                }
                 if (whole) {
                     float inv[HPT];
 #pragma unroll
