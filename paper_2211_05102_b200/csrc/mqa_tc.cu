@@ -1449,7 +1449,8 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
     // shared memory (the kernel checks on the device that the batch really is uniform; otherwise the pairs are
     // simply not used).  The host sees only Lmax, so the prediction assumes every sequence fills its cache.
     p.cluster = 1;
-    if (D == 256 && p.adaptive && (p.num_ctas % 2) == 0 &&
+    static const bool s_no_cluster = getenv("MQA_NO_CLUSTER") != nullptr;   // e.g. under a profiler that cannot launch clusters
+    if (!s_no_cluster && D == 256 && p.adaptive && (p.num_ctas % 2) == 0 &&
         uniform_ctas(p.B, (p.Lmax + kTileRows - 1) / kTileRows, p.num_ctas) == 2 * p.B) {
         static int s_pairs_fit[kMaxDevices] = {};   // 0 unknown, 1 yes, -1 no
         if (s_pairs_fit[dev] == 0) {
