@@ -1448,11 +1448,11 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
     // two halves: consecutive blocks then hold the halves of one sequence and merge them through distributed
     // shared memory (the kernel checks on the device that the batch really is uniform; otherwise the pairs are
     // simply not used).  The host sees only Lmax, so the prediction assumes every sequence fills its cache.
+    static int s_pairs_fit[kMaxDevices] = {};   // clusters of two on that device: 0 unknown, 1 they fit, -1 they do not
     p.cluster = 1;
     static const bool s_no_cluster = getenv("MQA_NO_CLUSTER") != nullptr;   // e.g. under a profiler that cannot launch clusters
     if (!s_no_cluster && D == 256 && p.adaptive && (p.num_ctas % 2) == 0 &&
         uniform_ctas(p.B, (p.Lmax + kTileRows - 1) / kTileRows, p.num_ctas) == 2 * p.B) {
-        static int s_pairs_fit[kMaxDevices] = {};   // 0 unknown, 1 yes, -1 no
         if (s_pairs_fit[dev] == 0) {
             cudaLaunchConfig_t probe = cfg;
             cudaLaunchAttribute pa[1];
@@ -1471,7 +1471,17 @@ cudaError_t launch_tc_t(const Params& p_in, cudaStream_t stream)
             p.cluster = 2;
         }
     }
-    return cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
+    e = cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
+    if (e != cudaSuccess && p.cluster == 2) {
+        // the occupancy query said the pairs fit, the launch disagrees (SMs taken by another context, say):
+        // clusters stay off on this device and the step runs with the global-memory merge
+        cudaGetLastError();
+        s_pairs_fit[dev] = -1;
+        cfg.numAttrs = 1;
+        p.cluster = 1;
+        e = cudaLaunchKernelEx(&cfg, mqa_tc_kernel<D, HP>, p, mc.mq, mc.mk, mc.mv, nslots);
+    }
+    return e;
 }
 
 }  // namespace
