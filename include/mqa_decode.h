@@ -37,6 +37,11 @@
  *     length limit (2147483647 = always both halves).
  *   - Thread safety: concurrent calls are safe when they use different
  *     workspaces.  Two calls sharing a workspace must be stream-ordered.
+ *   - Launches: the tensor-core path is ONE cooperative launch per call (its blocks wait for one another when
+ *     they merge a sequence that was cut, so all of them must be resident: at most one block per SM, and two
+ *     such calls on different streams run one after the other).  For some uniform batches the launch uses
+ *     thread-block clusters of two (environment variable MQA_NO_CLUSTER turns that off).  The launch can be
+ *     captured in a CUDA graph.  The FMA path enqueues two ordinary kernels.
  */
 #ifndef MQA_DECODE_H_
 #define MQA_DECODE_H_
