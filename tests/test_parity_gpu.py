@@ -295,3 +295,26 @@ def test_pair_mode_merges_halves_through_cluster_shared_memory(B, H, L):
     assert_close(run_gpu(q2, k2, v2, ln2, 1.0 / math.sqrt(D), workspace=ws),
                  ref.mqa_decode_ref(q2, k2, v2, ln2, 1.0 / math.sqrt(D)), "ragged under a cluster launch")
     assert int(ws[:32].view(torch.int32)[4]) == 0
+
+
+def test_cuda_graph_replay_in_pair_mode():
+    """The cluster launch of pair mode inside a CUDA graph: replays reproduce the eager result bit for bit."""
+    B, H, D, Lmax = 70, 16, 256, 512
+    dev = torch.device("cuda:0")
+    q, k, v, ln = make_custom(B, H, D, Lmax, seed=808, lengths=[512 - (i % 7) for i in range(B)])
+    qd, kd, vd, ld = q.to(dev), k.to(dev), v.to(dev), ln.to(dev)
+    out = torch.empty((B, H, D), dtype=torch.float32, device=dev)
+    ws = binding.alloc_workspace(B, H, D, Lmax)
+    binding.mqa_decode(qd, kd, vd, ld, out, 1 / 16, ws)
+    torch.cuda.synchronize()
+    eager = out.clone()
+    assert_close(eager.cpu(), ref.mqa_decode_ref(q, k, v, ln, 1 / 16), "eager")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.mqa_decode(qd, kd, vd, ld, out, 1 / 16, ws)
+    for _ in range(3):
+        out.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+    assert binding.mqa_check_status(ws) == binding.MQA_OK
