@@ -320,3 +320,28 @@ def test_cuda_graph_replay_in_pair_mode():
         torch.cuda.synchronize()
         assert torch.equal(out, eager)
     assert binding.mqa_check_status(ws) == binding.MQA_OK
+
+
+def test_two_streams_with_separate_workspaces():
+    """Steps enqueued alternately on two streams (separate workspaces): the cooperative launches, whose blocks
+    wait for one another, must not starve each other, and both results match the oracle."""
+    dev = torch.device("cuda:0")
+    B, H, D, Lmax = 40, 48, 256, 3000
+    qa, ka, va, la = make_custom(B, H, D, Lmax, seed=11, lengths=[3000 - 50 * i for i in range(B)])
+    qb, kb, vb, lb = make_custom(B, H, D, Lmax, seed=12, lengths=[1000 + 50 * i for i in range(B)])
+    ea = ref.mqa_decode_ref(qa, ka, va, la, 1 / 16)
+    eb = ref.mqa_decode_ref(qb, kb, vb, lb, 1 / 16)
+    a = [t.to(dev) for t in (qa, ka, va, la)]
+    b = [t.to(dev) for t in (qb, kb, vb, lb)]
+    oa = torch.empty((B, H, D), dtype=torch.float32, device=dev)
+    ob = torch.empty_like(oa)
+    wa, wb = binding.alloc_workspace(B, H, D, Lmax), binding.alloc_workspace(B, H, D, Lmax)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(30):
+        binding.mqa_decode(*a, oa, 1 / 16, wa, stream=s1)
+        binding.mqa_decode(*b, ob, 1 / 16, wb, stream=s2)
+    torch.cuda.synchronize()
+    assert binding.mqa_check_status(wa) == binding.MQA_OK and binding.mqa_check_status(wb) == binding.MQA_OK
+    assert_close(oa.cpu(), ea, "stream 1")
+    assert_close(ob.cpu(), eb, "stream 2")
