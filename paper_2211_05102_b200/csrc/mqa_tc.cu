@@ -1,5 +1,6 @@
 // Tensor-core multiquery decode kernel for sm_100a: TMA-staged K/V tiles, tcgen05
-// MMAs with accumulators in tensor memory, base-2 online softmax, partial writer.
+// MMAs with accumulators in tensor memory, base-2 online softmax, partial writer and
+// in-kernel merge.
 //
 // One persistent block per SM walks its run of 128-row K/V tiles (the flattened
 // schedule of mqa_common.cuh).  Each K/V tile is staged in shared memory ONCE by
@@ -9,12 +10,18 @@
 //     S^T[l, h] = K_tile[l, :] . Q[h, :]          M = 128 rows, N = HP, K = D
 //     O^T[d, h] += V_tile^T[d, l] . P^T[l, h]     M = 128 (per 128-wide half of D), N = HP, K = 128
 // S^T lives in tensor memory with one cache row per lane, so a softmax thread owns
-// one cache row and all heads.  The probabilities go back through shared memory
-// as bf16 hi + lo halves (two MMAs), which keeps ~16 bits of each probability.
+// one cache row and 16 heads (HP/16 independent warpgroups).  The probabilities go
+// back through shared memory as bf16 (plus the low-order bf16 half for sequences of
+// at most lo_max_len rows: two MMAs, ~16 bits of each probability).
 //
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (and tensor-memory owner),
-// warps 4-7 = softmax + segment epilogue.  Every wait is bounded; when one runs
-// out the block records MQA_ERR_TIMEOUT in the workspace header and leaves.
+// warp 2 = publisher of partial results, warps 4.. = softmax + segment epilogue.
+// A sequence that is cut between blocks is merged inside this launch: every block that
+// holds a part merges one slice of the output once all parts have arrived (global
+// memory, cooperative launch), or - for uniform batches cut into two halves, launched
+// as clusters of two - the halves are exchanged through distributed shared memory.
+// Every wait is bounded; when one runs out the block records MQA_ERR_TIMEOUT in the
+// workspace header and leaves.
 #include "mqa_common.cuh"
 
 #include <cuda.h>
