@@ -100,10 +100,16 @@ __device__ __forceinline__ float* ws_slot(unsigned char* ws, int B, int H, int D
     return reinterpret_cast<float*>(ws + slots_offset(B)) + (size_t)slot * slot_floats(H, D);
 }
 
-// First tile of block i's run.
-__host__ __device__ inline long long span_begin(int i, int T, int G) { return (long long)i * T / G; }
+// First tile of block i's run (0 <= i <= G).  The products are at most T*G: 32-bit arithmetic whenever that
+// fits (a 64-bit division is some hundred instructions, and these sit in every launch's prologue).
+__host__ __device__ inline long long span_begin(int i, int T, int G) {
+    if ((unsigned long long)(unsigned)T * (unsigned)G <= 0xffffffffull) return (long long)((unsigned)i * (unsigned)T / (unsigned)G);
+    return (long long)i * T / G;
+}
 // The block whose run contains tile g (0 <= g < T).
 __host__ __device__ inline int cta_of_tile(long long g, int T, int G) {
+    if ((unsigned long long)(unsigned)T * (unsigned)G + (unsigned)T <= 0xffffffffull)
+        return (int)((((unsigned)g + 1u) * (unsigned)G + (unsigned)T - 1u) / (unsigned)T) - 1;
     return (int)(((g + 1) * G + T - 1) / T) - 1;
 }
 

@@ -648,15 +648,19 @@ mqa_tc_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensor
     }
     const int N = (T > 0) ? (int)(misc.sched.g1 - misc.sched.g0) : 0;   // tiles of this block
     if (tid == 0) PROF_TS(1);
-    // Empty sequences own no tile: their output rows are zeroed here, round-robin over the blocks.
-    for (int b = cta; b < p.B; b += (int)gridDim.x) {
-        if (clamp_len(p.lengths[b], p.Lmax) == 0) {
-            for (int i = tid; i < H * D / 4; i += L::kThreads) {
-                const int h = (i * 4) / D;
-                *reinterpret_cast<float4*>(out_row(p, b, h) + (i * 4 - h * D)) = make_float4(0.f, 0.f, 0.f, 0.f);
+    // Empty sequences own no tile: their output rows are zeroed round-robin over the blocks, by the spare warp of a
+    // block that has tiles (off the path to the first load) or by all threads of a block that has none.
+    auto zero_empty_rows = [&](int t0, int nthr) {
+        for (int b = cta; b < p.B; b += (int)gridDim.x) {
+            if (clamp_len(p.lengths[b], p.Lmax) == 0) {
+                for (int i = t0; i < H * D / 4; i += nthr) {
+                    const int h = (i * 4) / D;
+                    *reinterpret_cast<float4*>(out_row(p, b, h) + (i * 4 - h * D)) = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
             }
         }
-    }
+    };
+    if (N == 0) zero_empty_rows(tid, L::kThreads);
 
     if (N > 0) {
         if (warp == 0) {
@@ -919,6 +923,8 @@ mqa_tc_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensor
 #endif
             PROF_END(kProfMmaTotal);
             if (lane == 0) PROF_TS(3);
+        } else if (warp == 3) {
+            zero_empty_rows(lane, 32);
         } else if (warp == 2) {
             // =============================== publisher of partial results ===============================
             // A block has at most two partial segments (the head of its run in slot 2*cta, the tail in 2*cta+1).
