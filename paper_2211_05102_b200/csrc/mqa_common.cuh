@@ -144,7 +144,6 @@ __host__ __device__ inline int uniform_ctas(int B, int nt, int G)
 
 struct SchedShared {
     int warp_sums[32];
-    int total;
     int b0;         // sequence that contains the first tile of this block's run
     int p0;         // global index of that sequence's first tile
     long long g0, g1;   // this block's run of tiles [g0, g1)
@@ -180,22 +179,17 @@ __device__ inline int schedule_prologue(const LenView lengths, int B, int Lmax,
     }
     if (lane == 31) sh.warp_sums[warp] = incl;
     uniform = __syncthreads_and(uniform) != 0;
-    if (warp == 0) {
-        int w = (lane < NTHREADS / 32) ? sh.warp_sums[lane] : 0;
-        int wi = w;
+    // every thread adds up the warp totals itself (one barrier and one serial step less than a second scan)
+    int T = 0, warp_offset = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, wi, o);
-            if (lane >= o) wi += t;
-        }
-        if (lane < NTHREADS / 32) sh.warp_sums[lane] = wi - w;   // exclusive warp offsets
-        if (lane == NTHREADS / 32 - 1) sh.total = wi;
+    for (int w = 0; w < NTHREADS / 32; ++w) {
+        const int s = sh.warp_sums[w];
+        T += s;
+        if (w < warp) warp_offset += s;
     }
-    __syncthreads();
-    const int T = sh.total;
     if (uniform) G = uniform_ctas(B, nt_first, G);    // identical in every thread of every block
     if (tid == 0) { sh.G = G; sh.pair = (uniform && G == 2 * B && (nt_first & 1) == 0) ? 1 : 0; }
-    int prefix = sh.warp_sums[warp] + incl - local;   // tiles before this thread's first sequence
+    int prefix = warp_offset + incl - local;          // tiles before this thread's first sequence
     if (T > 0 && cta < G) {
         const long long g0 = span_begin(cta, T, G);
         if (tid == 0) { sh.g0 = g0; sh.g1 = span_begin(cta + 1, T, G); }
